@@ -1,0 +1,116 @@
+/*
+ * attn.h — C interface of the B200 (sm_100a) fused attention forward with Rowmax weight maps.
+ *
+ * The library computes, for every batch b, query head h and query row i,
+ *
+ *     O[b,i,h,:] = v_descale * sum_j w_ij V[b,j,g(h),:] / sum_j w_ij,      LSE[b,h,i] = ln sum_j w_ij (+ anchor)
+ *
+ * over the keys j visible to row i, where the weight w_ij of a score is one of
+ *   exact : 2^x               softmax, Eq. m-exact (Sec. 3.1) / Eq. exact-attention (App. A)
+ *   pot   : 2^-min{K,floor(-x+1/2)}   Rowmax-PoT, Eq. rowmax-pot (App. A), K = K_max = 20
+ *   h15   : (1 + (n mod 2)/2) 2^floor(n/2), n = RNE(2x)   Rowmax-H15, Eq. m-h15 (Sec. 5.2) / Eq. h15 (App. B.1)
+ * and x is the score's base-two offset from the running row maximum of the online-softmax loop
+ * over key tiles (Sec. 5.2, App. B.1): x = s*c - m*c with c = softmax_scale*q_descale*k_descale*log2(e).
+ * In pot and h15 mode the result depends on the key-tile schedule, which attn_get_schedule reports.
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller.  The library never allocates,
+ *     frees or keeps them.  Calls are asynchronous on `stream` (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream) and do not synchronise the host.
+ *   - Return value: ATTN_OK (0) or a negative ATTN_ERR_* code.  Nothing is thrown, printed or aborted.
+ *   - Not thread-safe with respect to the per-process caches of tensor maps: call from one host
+ *     thread at a time.
+ */
+#ifndef ROWMAX_ATTN_H_
+#define ROWMAX_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { ATTN_W_EXACT = 0, ATTN_W_POT = 1, ATTN_W_H15 = 2 };
+enum { ATTN_IN_BF16 = 0, ATTN_IN_FP8_E4M3 = 1 };
+/* format of the probability tile P fed to the P.V contraction, as reported by attn_get_schedule */
+enum { ATTN_P_BF16 = 0, ATTN_P_E4M3 = 1, ATTN_P_E5M2 = 2 };
+
+enum {
+    ATTN_OK = 0,
+    ATTN_ERR_NULLPTR = -1,          /* a required pointer is NULL */
+    ATTN_ERR_BAD_SHAPE = -2,        /* B, H, S <= 0; Hq % Hkv != 0; unsupported D; size overflow */
+    ATTN_ERR_BAD_ENUM = -3,         /* weight_mode / in_dtype outside the enums above */
+    ATTN_ERR_MISALIGNED = -4,       /* q, k, v or o not 16-byte aligned */
+    ATTN_ERR_UNSUPPORTED_ARCH = -5, /* current device is not compute capability 10.x */
+    ATTN_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed; see attn_last_cuda_error */
+    ATTN_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired; see attn_device_status */
+    ATTN_ERR_UNSUPPORTED = -8,      /* valid arguments, combination not built (e.g. fp8 with D = 64) */
+    ATTN_ERR_BAD_VALUE = -9         /* softmax_scale or an fp8 descale is not positive and finite */
+};
+
+/*
+ * attn_fwd — fused attention forward (Sec. 5.2; App. B.1 for the loop the weight map lives in).
+ *
+ *   q            (B, Sq, Hq, D)   bf16, or e4m3 bytes when in_dtype = ATTN_IN_FP8_E4M3; D contiguous
+ *   k, v         (B, Sk, Hkv, D)  same storage type as q
+ *   o            (B, Sq, Hq, D)   bf16, written
+ *   lse          (B, Hq, Sq)      fp32, natural log, written; may be NULL
+ *   D            64 or 128 for bf16; 128 for fp8
+ *   causal       != 0: key j is visible to query i iff j <= i + Sk - Sq (aligned to the bottom-right
+ *                corner); a row that sees no key gets O = 0 and LSE = -inf
+ *   Hq, Hkv      query head h reads key/value head h / (Hq / Hkv)
+ *   softmax_scale  multiplies q.k before the softmax (natural-exponent units)
+ *   weight_mode  ATTN_W_EXACT / ATTN_W_POT / ATTN_W_H15
+ *   q/k/v_descale  per-tensor factors of the fp8 inputs (value = stored * descale); ignored for bf16
+ *
+ * All tensors are contiguous; q, k, v, o must be 16-byte aligned.  In pot/h15 mode LSE is the log
+ * of the approximated denominator.
+ */
+int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+             int B, int Hq, int Hkv, int Sq, int Sk, int D,
+             int causal, float softmax_scale, int weight_mode, int in_dtype,
+             float q_descale, float k_descale, float v_descale, void* stream);
+
+/*
+ * attn_weight_map — applies the weight map of `weight_mode` to n fp32 offsets with the same device
+ * function the fused kernel uses (Eq. m-exact / Eq. rowmax-pot / Eq. h15; the h15 input is clamped
+ * below at -126, App. B.1 "Implementation").  x and w are device arrays of n floats; they may alias.
+ * pot and h15 results are bit-exact by definition; exact uses the hardware ex2 approximation with
+ * subnormal results flushed to zero.
+ */
+int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* stream);
+
+/*
+ * attn_get_schedule — what a reference implementation must mirror to reproduce pot/h15 results
+ * (App. B "Semantic simulation": per-tile running maximum, tile of 128 keys, rescale rule).
+ * Host-only query, no CUDA call.  Any output pointer may be NULL.
+ *   tile_m, tile_n   query rows / keys per tile
+ *   kv_order         +1: key tiles visited in ascending order
+ *   rescale_tau      running-maximum adoption threshold in octaves (0 = the anchor is always current)
+ *   pot_kmax         K_max of Rowmax-PoT
+ *   p_format         ATTN_P_*; p_offset_log2: P is stored as weight * 2^p_offset_log2
+ */
+int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal,
+                      int* tile_m, int* tile_n, int* kv_order, float* rescale_tau,
+                      int* pot_kmax, int* p_format, int* p_offset_log2);
+
+/*
+ * attn_device_status — synchronises the current device and returns the sticky device-side status
+ * word: 0, or a code telling which bounded wait expired (role << 8 | barrier id).  A non-zero
+ * value means results of the affected launch are invalid.  attn_device_status_reset clears it.
+ * (No counterpart in the paper: safety net for the mbarrier/TMEM pipeline.)
+ */
+int attn_device_status(void);
+int attn_device_status_reset(void);
+
+/* Number of kernels this library has launched in this process (all entry points). */
+unsigned long long attn_launch_count(void);
+
+const char* attn_status_string(int status);
+int attn_last_cuda_error(void);     /* cudaError_t / CUresult of the last failing call, else 0 */
+const char* attn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROWMAX_ATTN_H_ */

@@ -1,0 +1,223 @@
+// C interface (include/attn.h): argument validation, TMA tensor maps, dispatch.  No torch types.
+#include "../../include/attn.h"
+#include "attn_kernel_common.cuh"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdint>
+
+namespace rowmax {
+cudaError_t launch_attn_fwd(int D, bool fp8, int mode, const CUtensorMap& tq, const CUtensorMap& tk,
+                            const CUtensorMap& tv, const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cudaStream_t stream);
+cudaError_t status_word_address(int** out);
+}  // namespace rowmax
+
+namespace {
+
+std::atomic<unsigned long long> g_launches{0};
+int g_last_cuda_error = 0;
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || sym == nullptr) {
+            g_last_cuda_error = static_cast<int>(e != cudaSuccess ? e : cudaErrorUnknown);
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// Tensor (B, S, H, D) with D contiguous, viewed innermost-first as (D, H, S, B); one box is
+// 128 bytes along D by 128 rows along S of a single head, 128-byte swizzled in shared memory.
+// Rows past S read as zero.
+int make_tile_map(CUtensorMap* map, const void* base, bool fp8, int B, int S, int H, int D) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return ATTN_ERR_CUDA;
+    const cuuint64_t es = fp8 ? 1 : 2;
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(S),
+                          static_cast<cuuint64_t>(B)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(D) * es, static_cast<cuuint64_t>(H) * D * es,
+                             static_cast<cuuint64_t>(S) * H * D * es};
+    cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / es), 1, 128, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = static_cast<int>(r);
+        return ATTN_ERR_CUDA;
+    }
+    return ATTN_OK;
+}
+
+int check_arch() {
+    static int cached_dev = -1, cached_ok = 0;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { g_last_cuda_error = e; return ATTN_ERR_CUDA; }
+    if (dev != cached_dev) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) { g_last_cuda_error = e; return ATTN_ERR_CUDA; }
+        cached_dev = dev;
+        cached_ok = (major == 10);
+    }
+    return cached_ok ? ATTN_OK : ATTN_ERR_UNSUPPORTED_ARCH;
+}
+
+int status_word(int** out) {
+    // one status word per device; looked up once per device
+    static int* words[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= 64) { g_last_cuda_error = e; return ATTN_ERR_CUDA; }
+    if (words[dev] == nullptr) {
+        e = rowmax::status_word_address(&words[dev]);
+        if (e != cudaSuccess) { g_last_cuda_error = e; words[dev] = nullptr; return ATTN_ERR_CUDA; }
+    }
+    *out = words[dev];
+    return ATTN_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+             int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
+             float k_descale, float v_descale, void* stream) {
+    if (!q || !k || !v || !o) return ATTN_ERR_NULLPTR;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15) return ATTN_ERR_BAD_ENUM;
+    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return ATTN_ERR_BAD_SHAPE;
+    if (D != 64 && D != 128) return ATTN_ERR_BAD_SHAPE;
+    if (B > 65535 || Hq > 65535) return ATTN_ERR_BAD_SHAPE;  // grid y/z limits
+    if (static_cast<long long>(Sq) + Sk >= (1ll << 30)) return ATTN_ERR_BAD_SHAPE;
+    const bool fp8 = in_dtype == ATTN_IN_FP8_E4M3;
+    if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return ATTN_ERR_BAD_VALUE;
+    if (fp8 && (!(q_descale > 0.f) || !(k_descale > 0.f) || !(v_descale > 0.f) || !std::isfinite(q_descale) ||
+                !std::isfinite(k_descale) || !std::isfinite(v_descale)))
+        return ATTN_ERR_BAD_VALUE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return ATTN_ERR_MISALIGNED;
+    if (fp8 && D != 128) return ATTN_ERR_UNSUPPORTED;
+    int rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+
+    rowmax::AttnParams p{};
+    p.o = o;
+    p.lse = lse;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
+    p.causal = causal != 0;
+    p.group = Hq / Hkv;
+    const double dq = fp8 ? static_cast<double>(q_descale) : 1.0;
+    const double dk = fp8 ? static_cast<double>(k_descale) : 1.0;
+    p.c = static_cast<float>(static_cast<double>(softmax_scale) * dq * dk * 1.4426950408889634074);
+    p.v_descale = fp8 ? v_descale : 1.0f;
+    rc = status_word(&p.status);
+    if (rc != ATTN_OK) return rc;
+
+    CUtensorMap tq, tk, tv;
+    if ((rc = make_tile_map(&tq, q, fp8, B, Sq, Hq, D)) != ATTN_OK) return rc;
+    if ((rc = make_tile_map(&tk, k, fp8, B, Sk, Hkv, D)) != ATTN_OK) return rc;
+    if ((rc = make_tile_map(&tv, v, fp8, B, Sk, Hkv, D)) != ATTN_OK) return rc;
+
+    cudaError_t e = rowmax::launch_attn_fwd(D, fp8, weight_mode, tq, tk, tv, p, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return e == cudaErrorInvalidValue ? ATTN_ERR_UNSUPPORTED : ATTN_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTN_OK;
+}
+
+int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* stream) {
+    if (n == 0) return ATTN_OK;
+    if (!x || !w) return ATTN_ERR_NULLPTR;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15) return ATTN_ERR_BAD_ENUM;
+    cudaError_t e = rowmax::launch_weight_map(x, w, n, weight_mode, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return ATTN_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTN_OK;
+}
+
+int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* tile_m, int* tile_n, int* kv_order,
+                      float* rescale_tau, int* pot_kmax, int* p_format, int* p_offset_log2) {
+    (void)causal;
+    if (D != 64 && D != 128) return ATTN_ERR_BAD_SHAPE;
+    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15) return ATTN_ERR_BAD_ENUM;
+    const bool fp8 = in_dtype == ATTN_IN_FP8_E4M3;
+    if (tile_m) *tile_m = rowmax::kTileM;
+    if (tile_n) *tile_n = rowmax::kTileN;
+    if (kv_order) *kv_order = +1;
+    if (rescale_tau) *rescale_tau = 0.0f;
+    if (pot_kmax) *pot_kmax = 20;
+    if (p_format) *p_format = !fp8 ? ATTN_P_BF16 : (weight_mode == ATTN_W_EXACT ? ATTN_P_E4M3 : ATTN_P_E5M2);
+    if (p_offset_log2) *p_offset_log2 = !fp8 ? 0 : (weight_mode == ATTN_W_EXACT ? 8 : 15);
+    return ATTN_OK;
+}
+
+int attn_device_status(void) {
+    int* word = nullptr;
+    int rc = status_word(&word);
+    if (rc != ATTN_OK) return rc;
+    int host = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&host, word, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return ATTN_ERR_CUDA; }
+    return host;
+}
+
+int attn_device_status_reset(void) {
+    int* word = nullptr;
+    int rc = status_word(&word);
+    if (rc != ATTN_OK) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemset(word, 0, sizeof(int));
+    if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return ATTN_ERR_CUDA; }
+    return ATTN_OK;
+}
+
+unsigned long long attn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* attn_status_string(int status) {
+    switch (status) {
+        case ATTN_OK: return "ok";
+        case ATTN_ERR_NULLPTR: return "null pointer";
+        case ATTN_ERR_BAD_SHAPE: return "bad shape";
+        case ATTN_ERR_BAD_ENUM: return "bad enum value";
+        case ATTN_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+        case ATTN_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+        case ATTN_ERR_CUDA: return "CUDA call failed";
+        case ATTN_ERR_TIMEOUT: return "device-side wait expired";
+        case ATTN_ERR_UNSUPPORTED: return "combination not built";
+        case ATTN_ERR_BAD_VALUE: return "scale or descale not positive and finite";
+        default: return "unknown status";
+    }
+}
+
+int attn_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* attn_version(void) { return "rowmax-attn-b200 0.1"; }
+
+}  // extern "C"

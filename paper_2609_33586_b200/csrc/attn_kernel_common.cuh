@@ -1,0 +1,29 @@
+// Parameters and small helpers shared by the attention kernels and the host launcher.
+#pragma once
+#include <cuda.h>
+#include <stdint.h>
+
+namespace rowmax {
+
+constexpr int kTileM = 128;  // query rows per tile
+constexpr int kTileN = 128;  // keys per tile
+
+enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2 };
+
+struct AttnParams {
+    void* o;          // (B,Sq,Hq,D) bf16
+    float* lse;       // (B,Hq,Sq) or nullptr
+    int B, Hq, Hkv, Sq, Sk;
+    int causal;
+    int group;        // Hq / Hkv
+    float c;          // softmax_scale * q_descale * k_descale * log2(e), rounded once to fp32
+    float v_descale;  // 1 for bf16
+    int* status;      // device-global sticky status word
+};
+
+// Status codes written by expired waits: role << 8 | barrier id.
+enum : int {
+    kRoleSerial = 1, kRoleLoad = 2, kRoleMma = 3, kRoleSoftmax = 4, kRoleCorr = 5, kRoleEpi = 6
+};
+
+}  // namespace rowmax

@@ -1,0 +1,60 @@
+// Device weight maps: exact (2^x), Rowmax-PoT (Eq. rowmax-pot) and Rowmax-H15 (Eq. h15), on fp32
+// base-two offsets.  The fused kernel and the sweep entry point use these same functions.
+#pragma once
+#include <stdint.h>
+
+namespace rowmax {
+
+constexpr int kPotKmax = 20;  // K_max of Rowmax-PoT (App. A, main point)
+
+// ---- exact: hardware ex2 (special-function unit), subnormal results flushed to zero.
+__device__ __forceinline__ float w_exact(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ---- Rowmax-H15 (Eq. h15; construction of App. B.1 "Implementation").
+// Input is the DOUBLED offset 2x.  After the clamp at -252, adding 2^23 + 2^22 as an fp32 value
+// rounds 2x to the nearest integer n (ties to even) and leaves 0x4B400000 + n in the bit pattern.
+constexpr float kH15Magic = 12582912.0f;       // 2^23 + 2^22, bit pattern 0x4B400000
+constexpr uint32_t kH15MagicBits = 0x4B400000u;
+
+__device__ __forceinline__ uint32_t h15_tbits(float x2) {
+    return __float_as_uint(fmaxf(x2, -252.0f) + kH15Magic);
+}
+// fp32 weight: shifting left by 22 drops the constant and puts bit 0 of n at the top of the
+// fraction and the rest in the exponent; adding the pattern of 1.0 supplies the bias:
+// bits = (n + 254) << 22, the value (1 + (n mod 2)/2) * 2^floor(n/2).
+__device__ __forceinline__ float h15_weight_from_tbits(uint32_t tbits) {
+    return __uint_as_float((tbits << 22) + 0x3F800000u);
+}
+__device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_from_tbits(h15_tbits(x2)); }
+// bf16 pattern of the same weight: the upper half of the fp32 pattern, (n + 254) << 6.  Exact.
+__device__ __forceinline__ uint32_t h15_bf16_from_tbits(uint32_t tbits) {
+    return ((tbits << 22) + 0x3F800000u) >> 16;
+}
+// e5m2 pattern of weight * 2^15: exponent field floor(n/2) + 30, top fraction bit n mod 2, i.e.
+// (n + 60) << 1.  Exact for n >= -58; below that the stored P flushes toward zero (relative to the
+// row maximum this is under 2^-29; the row sum still uses the fp32 weight).
+constexpr int kP8OffsetLog2 = 15;
+__device__ __forceinline__ uint32_t h15_e5m2_from_tbits(uint32_t tbits) {
+    int n60 = static_cast<int>(tbits - kH15MagicBits) + 4 * kP8OffsetLog2;
+    return static_cast<uint32_t>(max(n60, 0)) << 1;
+}
+
+// ---- Rowmax-PoT (Eq. rowmax-pot): d = min{K_max, floor(y + 1/2)}, y = -x, w = 2^-d.
+// floor(y + 1/2) without double rounding: one round-DOWN add of 2^22 + 64.5 leaves
+// 2^22 + floor(2 (y + 64.5)) / 2 exactly, whose integer part is floor(y + 1/2) + 64.
+__device__ __forceinline__ int pot_index(float x) {
+    float y = fminf(fmaxf(-x, -64.0f), 64.0f);
+    float t = __fadd_rd(y, 4194368.5f);
+    int twice = static_cast<int>(__float_as_uint(t) - 0x4A800000u);  // 2 * (t - 2^22)
+    int d = (twice >> 1) - 64;
+    return min(d, kPotKmax);
+}
+__device__ __forceinline__ float w_pot(float x) {
+    return __uint_as_float(static_cast<uint32_t>(127 - pot_index(x)) << 23);
+}
+
+}  // namespace rowmax

@@ -1,0 +1,113 @@
+"""GPU parity of the fused attention forward against the CPU oracle, through the C interface."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cpu_oracle as orc
+from paper_2609_33586_b200 import binding
+from paper_2609_33586_b200.inputs import WORKLOADS, Workload, make_inputs
+
+from parity_util import compare
+
+pytestmark = pytest.mark.gpu
+
+MODES = [orc.W_EXACT, orc.W_POT, orc.W_H15]
+
+
+@pytest.fixture(autouse=True)
+def _device_status_is_clean():
+    binding.device_status_reset()
+    yield
+    assert binding.device_status() == 0
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_config0_tiny_causal_every_row(mode):
+    st = compare(WORKLOADS[0], mode)
+    assert st["ok"], st
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("wl", [
+    Workload("d128_ragged", 2, 4, 2, 300, 300, 128, True, "bf16", 31),       # several tiles + ragged tail
+    Workload("d128_noncausal", 1, 2, 1, 257, 391, 128, False, "bf16", 32),   # Sq != Sk, not multiples of 128
+    Workload("d64_cross", 1, 4, 4, 130, 520, 64, True, "bf16", 33),          # bottom-right aligned mask
+    Workload("more_q_than_k", 1, 2, 2, 400, 144, 64, True, "bf16", 34),      # rows with no visible key
+    Workload("one_row", 1, 1, 1, 1, 1, 128, True, "bf16", 35),               # degenerate: single query and key
+    Workload("fp8_ragged", 2, 4, 2, 300, 428, 128, True, "fp8_e4m3", 36),
+    Workload("fp8_noncausal", 1, 2, 2, 256, 384, 128, False, "fp8_e4m3", 37),
+], ids=lambda w: w.name)
+def test_small_shapes(wl, mode):
+    st = compare(wl, mode)
+    assert st["ok"], st
+
+
+@pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_H15])
+def test_config1_gqa_peaked_rows(mode):
+    wl = WORKLOADS[1]
+    rows = np.unique(np.concatenate([np.arange(0, wl.Sq, 16), np.arange(128), np.arange(wl.Sq - 128, wl.Sq)]))
+    st = compare(wl, mode, rows=rows)
+    assert st["ok"], st
+
+
+def test_fully_masked_rows_give_zero_and_minus_infinity():
+    wl = Workload("masked", 1, 2, 2, 300, 100, 64, True, "bf16", 41)
+    inp = make_inputs(wl)
+    o, lse = binding.attn_fwd(inp.q.cuda(), inp.k.cuda(), inp.v.cuda(), causal=True,
+                              softmax_scale=wl.softmax_scale, weight_mode=orc.W_H15)
+    torch.cuda.synchronize()
+    assert torch.all(o[:, :200] == 0) and torch.all(torch.isneginf(lse[:, :, :200]))
+    assert torch.all(torch.isfinite(lse[:, :, 200:]))
+
+
+def test_run_twice_is_bitwise_deterministic():
+    wl = WORKLOADS[0].with_(Sq=512, Sk=512)
+    inp = make_inputs(wl)
+    q, k, v = inp.q.cuda(), inp.k.cuda(), inp.v.cuda()
+    a = binding.attn_fwd(q, k, v, causal=True, softmax_scale=wl.softmax_scale, weight_mode=orc.W_H15)
+    b = binding.attn_fwd(q, k, v, causal=True, softmax_scale=wl.softmax_scale, weight_mode=orc.W_H15)
+    torch.cuda.synchronize()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_h15_one_hot_values_expose_lattice_probabilities():
+    # One-hot value rows read the kernel's normalised probabilities back (App. B "Correctness gates").
+    S, D = 128, 128
+    wl = Workload("onehot", 1, 1, 1, S, S, D, True, "bf16", 42)
+    inp = make_inputs(wl)
+    inp.v = torch.eye(S, D).reshape(1, S, 1, D).to(torch.bfloat16)
+    o, _ = binding.attn_fwd(inp.q.cuda(), inp.k.cuda(), inp.v.cuda(), causal=True,
+                            softmax_scale=wl.softmax_scale, weight_mode=orc.W_H15)
+    p = o[0, :, 0].float().cpu().numpy()
+    assert np.all(np.triu(p, 1) == 0)                       # masked keys: probability zero
+    assert np.allclose(p.sum(axis=1), 1.0, atol=2e-2)       # bf16 storage of O
+    ex, _ = binding.attn_fwd(inp.q.cuda(), inp.k.cuda(), inp.v.cuda(), causal=True,
+                             softmax_scale=wl.softmax_scale, weight_mode=orc.W_EXACT)
+    pe = ex[0, :, 0].float().cpu().numpy()
+    big = np.tril(np.ones((S, S), bool)) & (pe > 1e-2)
+    ratio = np.log2(p[big] / pe[big])
+    assert np.all(np.abs(ratio) <= np.log2(1.5) + 0.03)     # +-0.585 octave, plus bf16 storage rounding
+
+
+def test_argument_errors_are_reported_without_launching():
+    before = binding.launch_count()
+    q = torch.zeros(1, 128, 2, 128, dtype=torch.bfloat16, device="cuda")
+    rc = binding.attn_fwd_raw(q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128,
+                              96, 1, 0.1, 0, 0, 1.0, 1.0, 1.0, None)
+    assert rc == -2                                       # D = 96
+    rc = binding.attn_fwd_raw(q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 3, 2, 128, 128,
+                              128, 1, 0.1, 0, 0, 1.0, 1.0, 1.0, None)
+    assert rc == -2                                       # Hq % Hkv
+    rc = binding.attn_fwd_raw(None, q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128, 128, 1, 0.1,
+                              0, 0, 1.0, 1.0, 1.0, None)
+    assert rc == -1
+    rc = binding.attn_fwd_raw(q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128,
+                              128, 1, 0.1, 5, 0, 1.0, 1.0, 1.0, None)
+    assert rc == -3
+    rc = binding.attn_fwd_raw(q.data_ptr() + 2, q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 64, 64,
+                              128, 1, 0.1, 0, 0, 1.0, 1.0, 1.0, None)
+    assert rc == -4
+    rc = binding.attn_fwd_raw(q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128,
+                              128, 1, -1.0, 0, 0, 1.0, 1.0, 1.0, None)
+    assert rc == -9
+    assert binding.launch_count() == before
