@@ -5,126 +5,119 @@
 //   S = Q K^T -> tile row maximum -> running maximum m (always adopted, threshold 0) ->
 //   x = s*c - m*c -> weight map -> row sum l and P (same weights) -> O = alpha*O + P V;
 // at the end O = v_descale * O / l and LSE = ln2 * (m*c + log2 l).
-#include "attn_kernel_common.cuh"
-#include "ptx.cuh"
-#include "weight_map.cuh"
+//
+// One CTA (16 warps) owns two query tiles of 128 rows of one (batch, head) and walks their key
+// tiles once, so every K/V tile staged in shared memory feeds four MMAs:
+//   warpgroup 0/1  softmax of query tile 0/1: one thread per row (no shuffles needed: a thread
+//                  reads its whole score row from TMEM), weight map, row sum, P written back to
+//                  TMEM over the S columns
+//   warpgroup 2    correction: rescales the O accumulators in TMEM when a running maximum moved,
+//                  and runs the epilogue
+//   warp 12        MMA issuer (one thread): S_t = Q_t K^T and O_t += P_t V on the tensor cores
+//   warp 13        TMA producer (one thread): Q once, then K/V through a ring of shared-memory slots
+// While warpgroup 0 works on S_0(j), the tensor cores compute P_1 V(j-1) and S_1(j), and vice versa.
+// TMEM columns: S_0/P_0 [0,128), S_1/P_1 [128,256), O_0 [256,384), O_1 [384,512).
+#include "attn_fwd_serial.cuh"
+#include "softmax_math.cuh"
 
-#include <cuda_bf16.h>
+#include <cstdlib>
 
 namespace rowmax {
 
 namespace {
 
 template <int D, bool FP8>
-struct TileCfg {
-    static constexpr int kElem = FP8 ? 1 : 2;
-    static constexpr int kRowBytes = D * kElem;
-    static constexpr int kBoxElems = 128 / kElem;           // one 128-byte swizzle row
-    static constexpr int kBoxes = kRowBytes / 128;          // boxes per tile along D
-    static constexpr int kBoxBytes = 128 * 128;             // 128 rows x 128 bytes
-    static constexpr int kTileBytes = kBoxes * kBoxBytes;   // 128 rows x D
-    static constexpr int kUmmaK = 32 / kElem;               // elements per MMA along K (32 bytes)
-    static constexpr int kQkSteps = D / kUmmaK;
-    static constexpr int kPvSteps = kTileN / kUmmaK;
-    static constexpr int kPCols = kTileN * kElem / 4;       // TMEM columns holding one P tile
-    static_assert(kRowBytes % 128 == 0, "row must be a whole number of 128-byte swizzle rows");
+struct WsCfg {
+    using C = TileCfg<D, FP8>;
+    static constexpr int kSlots = FP8 ? 8 : (D == 128 ? 4 : 8);  // K/V ring slots (one tile each)
+    static constexpr int kQBytes = 2 * C::kTileBytes;
+    static constexpr int kRingBytes = kSlots * C::kTileBytes;
+    static constexpr int kScaleOff = kQBytes + kRingBytes;        // float alpha[2][128]
+    static constexpr int kFinalOff = kScaleOff + 2 * 128 * 4;     // float2 (l, m)[2][128]
+    static constexpr int kBarOff = kFinalOff + 2 * 128 * 8;
+    static constexpr int kNumBars = 2 + 2 * kSlots + 6 * 2;
+    static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+    static constexpr int kSmemBytes = kMiscOff + 16 + 1024;       // + manual 1024-byte alignment slack
+    static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
 };
 
-__device__ __forceinline__ uint32_t pack_bf16_rn(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-__device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
-    uint16_t r;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
+__device__ __forceinline__ void reg_dec_48() { asm volatile("setmaxnreg.dec.sync.aligned.u32 48;"); }
+__device__ __forceinline__ void reg_dec_80() { asm volatile("setmaxnreg.dec.sync.aligned.u32 80;"); }
+__device__ __forceinline__ void reg_inc_192() { asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); }
 
-// exact-mode fp8 path stores P = w * 2^8 in e4m3 (largest value 256 <= 448)
-constexpr int kP8ExactOffsetLog2 = 8;
-
-// Turns 32 consecutive scores of one row into weights: returns their sum and writes the packed P
-// words (16 words of 2 bf16, or 8 words of 4 fp8).  `limit` = first masked column of the chunk.
-template <bool FP8, int MODE>
-__device__ __forceinline__ float weights_chunk32(const uint32_t (&sraw)[32], float c_eff, float mc_eff,
-                                                 int limit, uint32_t* pw) {
-    float acc0 = 0.f, acc1 = 0.f;
-    uint32_t pb[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const float s = __uint_as_float(sraw[i]);
-        const bool masked = i >= limit;
-        float w;
-        uint32_t bits;  // P pattern: bf16 in the low 16 bits, or an fp8 byte
-        if constexpr (MODE == kExact) {
-            w = w_exact(fmaf(s, c_eff, -mc_eff));  // masked scores are -inf -> weight 0
-            bits = 0;
-        } else if constexpr (MODE == kH15) {
-            const uint32_t tb = h15_tbits(fmaf(s, c_eff, -mc_eff));  // c_eff = 2c: doubled input
-            w = h15_weight_from_tbits(tb);
-            bits = FP8 ? h15_e5m2_from_tbits(tb) : (__float_as_uint(w) >> 16);
-        } else {
-            const int d = pot_index(fmaf(s, c_eff, -mc_eff));
-            w = __uint_as_float(static_cast<uint32_t>(127 - d) << 23);
-            bits = FP8 ? static_cast<uint32_t>(15 + kP8OffsetLog2 - d) << 2 : (__float_as_uint(w) >> 16);
-        }
-        if constexpr (MODE != kExact) {
-            if (masked) { w = 0.f; bits = 0; }
-        }
-        pb[i] = (MODE == kExact) ? __float_as_uint(w) : bits;
-        if (i & 1) acc1 += w; else acc0 += w;
-    }
-    if constexpr (!FP8) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            if constexpr (MODE == kExact)
-                pw[i] = pack_bf16_rn(__uint_as_float(pb[2 * i]), __uint_as_float(pb[2 * i + 1]));
-            else
-                pw[i] = pb[2 * i] | (pb[2 * i + 1] << 16);
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if constexpr (MODE == kExact)
-                pw[i] = pack_e4m3x2(__uint_as_float(pb[4 * i]), __uint_as_float(pb[4 * i + 1])) |
-                        (pack_e4m3x2(__uint_as_float(pb[4 * i + 2]), __uint_as_float(pb[4 * i + 3])) << 16);
-            else
-                pw[i] = pb[4 * i] | (pb[4 * i + 1] << 8) | (pb[4 * i + 2] << 16) | (pb[4 * i + 3] << 24);
-        }
-    }
-    return acc0 + acc1;
-}
+enum BarId : int { kBarQ = 0, kBarKvFull = 1, kBarKvEmpty = 2, kBarSFull = 3, kBarPFull = 4, kBarOFull = 5,
+                   kBarScale = 6, kBarORescaled = 7, kBarFinal = 8 };
 
 }  // namespace
 
-// ------------------------------------------------------------------------------------------------
-// Serial kernel: one CTA of 128 threads per (query tile, head, batch); thread t owns query row t.
-// Every step waits for the previous one (no overlap).  It fixes the data layouts and descriptors.
-// ------------------------------------------------------------------------------------------------
 template <int D, bool FP8, int MODE>
-__global__ void __launch_bounds__(128, 1)
-attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                       const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+__global__ void __launch_bounds__(512, 1)
+attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
     using C = TileCfg<D, FP8>;
+    using W = WsCfg<D, FP8>;
+    constexpr int NS = W::kSlots;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    const uint32_t sQ = smem_u32(smem), sK = sQ + C::kTileBytes, sV = sK + C::kTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 3 * C::kTileBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    const uint32_t bar_q = smem_u32(&bars[0]), bar_kv = smem_u32(&bars[1]), bar_mma = smem_u32(&bars[2]);
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const uint32_t sQ = smem_u32(smem);
+    const uint32_t sRing = sQ + W::kQBytes;
+    float* sScale = reinterpret_cast<float*>(smem + W::kScaleOff);
+    float2* sFinal = reinterpret_cast<float2*>(smem + W::kFinalOff);
+    const uint32_t bar0 = smem_u32(smem + W::kBarOff);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + W::kMiscOff);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + W::kMiscOff + 4);
     const WaitCtx wctx{abort_flag, p.status};
 
+    // barrier addresses
+    auto bar_q = [&](int t) { return bar0 + 8u * t; };
+    auto bar_kv_full = [&](int s) { return bar0 + 8u * (2 + s); };
+    auto bar_kv_empty = [&](int s) { return bar0 + 8u * (2 + NS + s); };
+    auto bar_x = [&](int which, int t) { return bar0 + 8u * (2 + 2 * NS + 2 * which + t); };
+    auto bar_s_full = [&](int t) { return bar_x(0, t); };      // MMA -> softmax: S_t(j) is in TMEM
+    auto bar_p_full = [&](int t) { return bar_x(1, t); };      // softmax -> MMA: P_t(j) is in TMEM
+    auto bar_o_full = [&](int t) { return bar_x(2, t); };      // MMA -> correction: P_t V(j) accumulated
+    auto bar_scale = [&](int t) { return bar_x(3, t); };       // softmax -> correction: alpha_t(j) in smem
+    auto bar_o_rescaled = [&](int t) { return bar_x(4, t); };  // correction -> MMA: O_t rescaled for tile j
+    auto bar_final = [&](int t) { return bar_x(5, t); };       // softmax -> correction: (l, m) in smem
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
+
+    // work item: heaviest query tiles first (they have the most key tiles under a causal mask)
+    const int n_pairs = (p.Sq + 2 * kTileM - 1) / (2 * kTileM);
+    const int bh = p.Hq * p.B;
+    const int pair = n_pairs - 1 - static_cast<int>(blockIdx.x) / bh;
+    const int rem = static_cast<int>(blockIdx.x) % bh;
+    const int h = rem % p.Hq, b = rem / p.Hq, hk = h / p.group;
+    const int shift = p.Sk - p.Sq;
+    int q0t[2], n_t[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        q0t[t] = pair * 2 * kTileM + t * kTileM;
+        int kv_end = p.causal ? min(p.Sk, q0t[t] + kTileM + shift) : p.Sk;
+        n_t[t] = (q0t[t] < p.Sq && kv_end > 0) ? (kv_end + kTileN - 1) / kTileN : 0;
+    }
+    const int n_max = max(n_t[0], n_t[1]);
+
     if (tid == 0) {
-        mbar_init(bar_q, 1);
-        mbar_init(bar_kv, 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_q(0), 1);
+        mbar_init(bar_q(1), 1);
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_kv_full(s), 1);
+            mbar_init(bar_kv_empty(s), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar_s_full(t), 1);
+            mbar_init(bar_p_full(t), 128);
+            mbar_init(bar_o_full(t), 1);
+            mbar_init(bar_scale(t), 128);
+            mbar_init(bar_o_rescaled(t), 128);
+            mbar_init(bar_final(t), 128);
+        }
         *abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0);
         fence_mbar_init();
     }
-    constexpr uint32_t kTmemCols = 256;
-    if (warp == 0) {
+    constexpr uint32_t kTmemCols = 512;
+    if (warp == 12) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -132,167 +125,258 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tmem_S = tmem, tmem_P = tmem, tmem_O = tmem + 128;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-
-    const int q0 = blockIdx.x * kTileM, h = blockIdx.y, b = blockIdx.z, hk = h / p.group;
-    const int shift = p.Sk - p.Sq;
-    int kv_end = p.Sk;
-    if (p.causal) kv_end = min(p.Sk, q0 + kTileM + shift);
-    const int n_tiles = kv_end > 0 ? (kv_end + kTileN - 1) / kTileN : 0;
-    const int row = q0 + tid;
-    const int row_limit = p.causal ? min(p.Sk, row + shift + 1) : p.Sk;  // visible keys of this row
+    auto tmem_S = [&](int t) { return tmem + 128u * t; };
+    auto tmem_O = [&](int t) { return tmem + 256u + 128u * t; };
 
     constexpr uint32_t fmt_ab = FP8 ? kFmtE4M3 : kFmtBF16;
     constexpr uint32_t fmt_p = FP8 ? (MODE == kExact ? kFmtE4M3 : kFmtE5M2) : kFmtBF16;
     constexpr uint32_t idesc_s = umma_idesc(fmt_ab, fmt_ab, false, false, kTileM, kTileN);
     constexpr uint32_t idesc_pv = umma_idesc(fmt_p, fmt_ab, false, true, kTileM, D);
-
-    auto load_kv = [&](int j) {
-        mbar_arrive_expect_tx(bar_kv, 2 * C::kTileBytes);
-#pragma unroll
-        for (int bx = 0; bx < C::kBoxes; ++bx) {
-            tma_load_4d(sK + bx * C::kBoxBytes, &tmK, bar_kv, bx * C::kBoxElems, hk, j * kTileN, b);
-            tma_load_4d(sV + bx * C::kBoxBytes, &tmV, bar_kv, bx * C::kBoxElems, hk, j * kTileN, b);
-        }
-    };
-
-    if (tid == 0 && n_tiles > 0 && !*abort_flag) {
-        mbar_arrive_expect_tx(bar_q, C::kTileBytes);
-#pragma unroll
-        for (int bx = 0; bx < C::kBoxes; ++bx)
-            tma_load_4d(sQ + bx * C::kBoxBytes, &tmQ, bar_q, bx * C::kBoxElems, h, q0, b);
-        load_kv(0);
-    }
-
-    // exact: x = s*c - m*c (+ the fp8 P offset);  h15: doubled input 2x = s*(2c) - m*(2c)
-    const float c_eff = (MODE == kH15) ? 2.0f * p.c : p.c;
     const float x_bias = (FP8 && MODE == kExact) ? static_cast<float>(kP8ExactOffsetLog2) : 0.0f;
-    float m_run = -INFINITY, l_run = 0.f;
-    uint32_t ph_mma = 0;
 
-    for (int j = 0; j < n_tiles; ++j) {
-        if (tid == 0 && !*abort_flag) {
-            if (j == 0) mbar_wait(bar_q, 0, wctx, (kRoleSerial << 8) | 0);
-            mbar_wait(bar_kv, j & 1, wctx, (kRoleSerial << 8) | 1);
-            tc_fence_after();
+    if (wg == 3) {
+        reg_dec_48();
+        if (warp == 13 && lane == 0) {
+            // ------------------------------------------------------------ TMA producer
+            auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, uint32_t bar, int head, int row0) {
+                mbar_arrive_expect_tx(bar, C::kTileBytes);
+#pragma unroll
+                for (int bx = 0; bx < C::kBoxes; ++bx)
+                    tma_load_4d(dst + bx * C::kBoxBytes, tm, bar, bx * C::kBoxElems, head, row0, b);
+            };
             if (!*abort_flag) {
+                if (n_t[0] > 0) load_tile(&tmQ, sQ, bar_q(0), h, q0t[0]);
+                for (int j = 0; j < n_max; ++j) {
+#pragma unroll
+                    for (int kv = 0; kv < 2; ++kv) {
+                        const int idx = 2 * j + kv, slot = idx % NS, use = idx / NS;
+                        mbar_wait(bar_kv_empty(slot), (use & 1) ^ 1, wctx, (kRoleLoad << 8) | kBarKvEmpty);
+                        if (*abort_flag) break;
+                        load_tile(kv == 0 ? &tmK : &tmV, sRing + slot * C::kTileBytes, bar_kv_full(slot), hk, j * kTileN);
+                        if (j == 0 && kv == 0 && n_t[1] > 0) load_tile(&tmQ, sQ + C::kTileBytes, bar_q(1), h, q0t[1]);
+                    }
+                }
+            }
+        } else if (warp == 12 && lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
+            auto issue_s = [&](int t, uint32_t sK) {
+                const uint32_t q = sQ + t * C::kTileBytes;
 #pragma unroll
                 for (int ks = 0; ks < C::kQkSteps; ++ks) {
                     const uint32_t off = (ks / 4) * C::kBoxBytes + (ks % 4) * 32;
-                    umma_ss<FP8>(tmem_S, umma_desc_sw128(sQ + off, 16, 1024), umma_desc_sw128(sK + off, 16, 1024),
+                    umma_ss<FP8>(tmem_S(t), umma_desc_sw128(q + off, 16, 1024), umma_desc_sw128(sK + off, 16, 1024),
                                  idesc_s, ks > 0);
                 }
-                umma_commit(bar_mma);
+            };
+            auto issue_pv = [&](int t, uint32_t sV, bool accumulate) {
+#pragma unroll
+                for (int ks = 0; ks < C::kPvSteps; ++ks) {
+                    const uint64_t bdesc = umma_desc_sw128(sV + ks * C::kUmmaK * 128, C::kBoxBytes, 1024);
+                    umma_ts<FP8>(tmem_O(t), tmem_S(t) + ks * 8, bdesc, idesc_pv, (accumulate || ks > 0) ? 1u : 0u);
+                }
+            };
+            auto slot_addr = [&](int idx) { return sRing + (idx % NS) * C::kTileBytes; };
+            auto wait_full = [&](int idx) {
+                mbar_wait(bar_kv_full(idx % NS), (idx / NS) & 1, wctx, (kRoleMma << 8) | kBarKvFull);
+            };
+            if (n_max > 0) {
+                wait_full(0);
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (n_t[t] > 0) {
+                        mbar_wait(bar_q(t), 0, wctx, (kRoleMma << 8) | kBarQ);
+                        tc_fence_after();
+                        if (!*abort_flag) issue_s(t, slot_addr(0));
+                        umma_commit(bar_s_full(t));
+                    }
+                }
+                umma_commit(bar_kv_empty(0));
+                for (int j = 0; j < n_max; ++j) {
+                    wait_full(2 * j + 1);
+                    bool k_ready = false;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (j < n_t[t]) {
+                            mbar_wait(bar_p_full(t), j & 1, wctx, (kRoleMma << 8) | kBarPFull);
+                            mbar_wait(bar_o_rescaled(t), j & 1, wctx, (kRoleMma << 8) | kBarORescaled);
+                            tc_fence_after();
+                            if (!*abort_flag) issue_pv(t, slot_addr(2 * j + 1), j > 0);
+                            umma_commit(bar_o_full(t));
+                        }
+                        if (j + 1 < n_t[t]) {
+                            if (!k_ready) {
+                                wait_full(2 * j + 2);
+                                tc_fence_after();
+                                k_ready = true;
+                            }
+                            if (!*abort_flag) issue_s(t, slot_addr(2 * j + 2));
+                            umma_commit(bar_s_full(t));
+                        }
+                    }
+                    umma_commit(bar_kv_empty((2 * j + 1) % NS));
+                    if (j + 1 < n_max) umma_commit(bar_kv_empty((2 * j + 2) % NS));
+                }
             }
         }
-        mbar_wait(bar_mma, ph_mma, wctx, (kRoleSerial << 8) | 2);
-        ph_mma ^= 1;
-        __syncwarp();
-        tc_fence_after();
-
-        uint32_t s[4][32];
+    } else if (wg == 2) {
+        // ---------------------------------------------------------------- correction + epilogue
+        reg_dec_80();
+        const int r = tid & 127;
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        for (int j = 0; j < n_max; ++j) {
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) tmem_ld32(tmem_S + lane_base + cc * 32, s[cc]);
-        tmem_wait_ld();
-
-        const int col_limit = row_limit - j * kTileN;  // columns >= col_limit are masked
-        float m_t = -INFINITY;
-        if (col_limit < kTileN) {
+            for (int t = 0; t < 2; ++t) {
+                if (j < n_t[t]) {
+                    mbar_wait(bar_scale(t), j & 1, wctx, (kRoleCorr << 8) | kBarScale);
+                    const float alpha = sScale[t * 128 + r];
+                    if (j > 0) {
+                        mbar_wait(bar_o_full(t), (j - 1) & 1, wctx, (kRoleCorr << 8) | kBarOFull);
+                        __syncwarp();
+                        tc_fence_after();
+                        if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc)
+                            for (int cc = 0; cc < D / 32; ++cc) {
+                                uint32_t o[32];
+                                tmem_ld32(tmem_O(t) + lane_base + cc * 32, o);
+                                tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (cc * 32 + i >= col_limit) s[cc][i] = __float_as_uint(-INFINITY);
+                                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                tmem_st32(tmem_O(t) + lane_base + cc * 32, o);
+                            }
+                            tmem_wait_st();
+                        }
+                        tc_fence_before();
+                    }
+                    mbar_arrive(bar_o_rescaled(t));
+                }
+            }
         }
+        // epilogue: O = v_descale * acc / l (undoing the P offset), LSE = ln2 * (m c + log2 l)
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-            for (int i = 0; i < 32; ++i) m_t = fmaxf(m_t, __uint_as_float(s[cc][i]));
-
-        const float m_new = fmaxf(m_run, m_t);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = ex2_approx((m_run - m_use) * p.c);
-        const float mc_eff = m_use * c_eff - x_bias;
-        m_run = m_new;
-
-        // every S column is in registers now, so P may overwrite the S columns
-        float l_tile = 0.f;
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-            uint32_t pw[16];
-            l_tile += weights_chunk32<FP8, MODE>(s[cc], c_eff, mc_eff, col_limit - cc * 32, pw);
-            if constexpr (FP8) tmem_st8(tmem_P + lane_base + cc * 8, pw);
-            else tmem_st16(tmem_P + lane_base + cc * 16, pw);
-        }
-        l_run = l_run * alpha + l_tile;
-
-        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+        for (int t = 0; t < 2; ++t) {
+            const int row = q0t[t] + r;
+            if (q0t[t] >= p.Sq) continue;
+            float l_run = 0.f, m_run = -INFINITY;
+            if (n_t[t] > 0) {
+                mbar_wait(bar_final(t), 0, wctx, (kRoleEpi << 8) | kBarFinal);
+                const float2 lm = sFinal[t * 128 + r];
+                l_run = lm.x;
+                m_run = lm.y;
+                mbar_wait(bar_o_full(t), (n_t[t] - 1) & 1, wctx, (kRoleEpi << 8) | kBarOFull);
+                __syncwarp();
+                tc_fence_after();
+            }
+            const bool has_keys = l_run > 0.f;
+            const float p_unscale = (FP8 && MODE != kExact) ? exp2f(-static_cast<float>(kP8OffsetLog2)) : 1.0f;
+            const float inv = has_keys ? p.v_descale * p_unscale / l_run : 0.f;
+            if (row < p.Sq && p.lse != nullptr) {
+                const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - x_bias) : -INFINITY;
+                p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.Sq + row] = lse;
+            }
+            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
+                                  ((static_cast<size_t>(b) * p.Sq + row) * p.Hq + h) * D;
 #pragma unroll
             for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t o[32];
-                tmem_ld32(tmem_O + lane_base + cc * 32, o);
-                tmem_wait_ld();
+                if (n_t[t] > 0) {
+                    tmem_ld32(tmem_O(t) + lane_base + cc * 32, o);
+                    tmem_wait_ld();
+                } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                tmem_st32(tmem_O + lane_base + cc * 32, o);
+                    for (int i = 0; i < 32; ++i) o[i] = 0;
+                }
+                if (row < p.Sq) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 pk;
+                        pk.x = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
+                        pk.y = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
+                        pk.z = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
+                        pk.w = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + cc * 32 + v4 * 8) = pk;
+                    }
+                }
             }
         }
-        tmem_wait_st();
-        tc_fence_before();
-        __syncthreads();
-
-        if (tid == 0 && !*abort_flag) {
+    } else {
+        // ---------------------------------------------------------------- softmax of query tile t
+        reg_inc_192();
+        const int t = wg;
+        const int r = tid & 127;
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_S(t) + lane_base;
+        const int q0 = t == 0 ? q0t[0] : q0t[1];
+        const int nt = t == 0 ? n_t[0] : n_t[1];
+        const int row = q0 + r;
+        const int row_limit = p.causal ? min(p.Sk, row + shift + 1) : p.Sk;  // visible keys of this row
+        // first key index that some row of this tile cannot see (tile-uniform)
+        const int tile_limit = p.causal ? min(p.Sk, q0 + shift + 1) : p.Sk;
+        const float c_eff = (MODE == kH15) ? 2.0f * p.c : p.c;
+        float m_run = -INFINITY, l_run = 0.f;
+        for (int j = 0; j < nt; ++j) {
+            mbar_wait(bar_s_full(t), j & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);
+            __syncwarp();
             tc_fence_after();
+            uint32_t s[4][32];
 #pragma unroll
-            for (int ks = 0; ks < C::kPvSteps; ++ks) {
-                const uint64_t bdesc = umma_desc_sw128(sV + ks * C::kUmmaK * 128, C::kBoxBytes, 1024);
-                umma_ts<FP8>(tmem_O, tmem_P + ks * 8, bdesc, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-            }
-            umma_commit(bar_mma);
-        }
-        mbar_wait(bar_mma, ph_mma, wctx, (kRoleSerial << 8) | 3);
-        ph_mma ^= 1;
-        if (tid == 0 && j + 1 < n_tiles && !*abort_flag) load_kv(j + 1);
-        __syncwarp();
-    }
-    tc_fence_after();
-
-    // epilogue: O = v_descale * acc / l (undoing the P offset), LSE = ln2 * (m c + log2 l)
-    const bool has_keys = l_run > 0.f;
-    const float p_unscale = (FP8 && MODE != kExact) ? exp2f(-static_cast<float>(kP8OffsetLog2)) : 1.0f;
-    const float inv = has_keys ? p.v_descale * p_unscale / l_run : 0.f;
-    if (row < p.Sq && p.lse != nullptr) {
-        const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - x_bias) : -INFINITY;
-        p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.Sq + row] = lse;
-    }
-    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
-                          ((static_cast<size_t>(b) * p.Sq + row) * p.Hq + h) * D;
-#pragma unroll
-    for (int cc = 0; cc < D / 32; ++cc) {
-        uint32_t o[32];
-        if (n_tiles > 0) {
-            tmem_ld32(tmem_O + lane_base + cc * 32, o);
+            for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, s[cc]);
             tmem_wait_ld();
-        } else {
+
+            const bool masked_tile = (j + 1) * kTileN > tile_limit;
+            const int col_limit = row_limit - j * kTileN;
+            if (masked_tile) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = 0;
-        }
-        if (row < p.Sq) {
+                for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-            for (int v4 = 0; v4 < 4; ++v4) {
-                uint4 pk;
-                pk.x = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
-                pk.y = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
-                pk.z = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
-                pk.w = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
-                *reinterpret_cast<uint4*>(orow + cc * 32 + v4 * 8) = pk;
+                    for (int i = 0; i < 32; ++i)
+                        if (cc * 32 + i >= col_limit) s[cc][i] = __float_as_uint(-INFINITY);
             }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(s[cc][i]));
+            const float m_t = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            const float m_new = fmaxf(m_run, m_t);
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            const float alpha = ex2_approx((m_run - m_use) * p.c);
+            const float mc_eff = m_use * c_eff - x_bias;
+            m_run = m_new;
+            sScale[t * 128 + r] = alpha;
+            mbar_arrive(bar_scale(t));
+
+            float l_tile = 0.f;
+            if (masked_tile) {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t pw[16];
+                    l_tile += weights_chunk32<FP8, MODE, true>(s[cc], c_eff, mc_eff, col_limit - cc * 32, pw);
+                    if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
+                    else tmem_st16(tS + cc * 16, pw);
+                }
+            } else {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t pw[16];
+                    l_tile += weights_chunk32<FP8, MODE, false>(s[cc], c_eff, mc_eff, 32, pw);
+                    if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
+                    else tmem_st16(tS + cc * 16, pw);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p_full(t));
+            l_run = l_run * alpha + l_tile;
+        }
+        if (nt > 0) {
+            sFinal[t * 128 + r] = make_float2(l_run, m_run);
+            mbar_arrive(bar_final(t));
         }
     }
+
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 12) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -315,13 +399,33 @@ static cudaError_t launch_serial(const CUtensorMap& tq, const CUtensorMap& tk, c
     return cudaGetLastError();
 }
 
+template <int D, bool FP8, int MODE>
+static cudaError_t launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                             const AttnParams& p, cudaStream_t stream) {
+    using W = WsCfg<D, FP8>;
+    static const bool serial = std::getenv("ROWMAX_ATTN_SERIAL") != nullptr;
+    if (serial) return launch_serial<D, FP8, MODE>(tq, tk, tv, p, stream);
+    auto kern = attn_fwd_ws_kernel<D, FP8, MODE>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, W::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const long long n_pairs = (p.Sq + 2 * kTileM - 1) / (2 * kTileM);
+    const long long blocks = n_pairs * p.Hq * p.B;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), 512, W::kSmemBytes, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError();
+}
+
 template <int D, bool FP8>
 static cudaError_t dispatch_mode(int mode, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                  const AttnParams& p, cudaStream_t stream) {
     switch (mode) {
-        case kExact: return launch_serial<D, FP8, kExact>(tq, tk, tv, p, stream);
-        case kPot: return launch_serial<D, FP8, kPot>(tq, tk, tv, p, stream);
-        default: return launch_serial<D, FP8, kH15>(tq, tk, tv, p, stream);
+        case kExact: return launch_ws<D, FP8, kExact>(tq, tk, tv, p, stream);
+        case kPot: return launch_ws<D, FP8, kPot>(tq, tk, tv, p, stream);
+        default: return launch_ws<D, FP8, kH15>(tq, tk, tv, p, stream);
     }
 }
 
