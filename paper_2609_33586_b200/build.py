@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libattn_b200.so"
 SOURCES = ["api.cu", "attn_fwd_sm100.cu"]
-HEADERS = ["ptx.cuh", "weight_map.cuh", "attn_kernel_common.cuh", "../../include/attn.h"]
+HEADERS = ["ptx.cuh", "weight_map.cuh", "attn_kernel_common.cuh", "softmax_math.cuh", "../../include/attn.h"]
 
 
 def _nvcc() -> str:

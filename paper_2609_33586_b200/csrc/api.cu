@@ -130,6 +130,7 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
     const double dk = fp8 ? static_cast<double>(k_descale) : 1.0;
     p.c = static_cast<float>(static_cast<double>(softmax_scale) * dq * dk * 1.4426950408889634074);
     p.v_descale = fp8 ? v_descale : 1.0f;
+    p.two22 = 1u << 22;
     rc = status_word(&p.status);
     if (rc != ATTN_OK) return rc;
 

@@ -17,10 +17,7 @@
 //   warp 13        TMA producer (one thread): Q once, then K/V through a ring of shared-memory slots
 // While warpgroup 0 works on S_0(j), the tensor cores compute P_1 V(j-1) and S_1(j), and vice versa.
 // TMEM columns: S_0/P_0 [0,128), S_1/P_1 [128,256), O_0 [256,384), O_1 [384,512).
-#include "attn_fwd_serial.cuh"
 #include "softmax_math.cuh"
-
-#include <cstdlib>
 
 namespace rowmax {
 
@@ -132,7 +129,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     constexpr uint32_t fmt_p = FP8 ? (MODE == kExact ? kFmtE4M3 : kFmtE5M2) : kFmtBF16;
     constexpr uint32_t idesc_s = umma_idesc(fmt_ab, fmt_ab, false, false, kTileM, kTileN);
     constexpr uint32_t idesc_pv = umma_idesc(fmt_p, fmt_ab, false, true, kTileM, D);
-    const float x_bias = (FP8 && MODE == kExact) ? static_cast<float>(kP8ExactOffsetLog2) : 0.0f;
+    constexpr float p_off = static_cast<float>(PFormat<FP8, MODE>::kOffLog2);  // log2 of the P / row-sum scale
 
     if (wg == 3) {
         reg_dec_48();
@@ -267,10 +264,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tc_fence_after();
             }
             const bool has_keys = l_run > 0.f;
-            const float p_unscale = (FP8 && MODE != kExact) ? exp2f(-static_cast<float>(kP8OffsetLog2)) : 1.0f;
-            const float inv = has_keys ? p.v_descale * p_unscale / l_run : 0.f;
+            const float inv = has_keys ? p.v_descale / l_run : 0.f;
             if (row < p.Sq && p.lse != nullptr) {
-                const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - x_bias) : -INFINITY;
+                const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - p_off) : -INFINITY;
                 p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.Sq + row] = lse;
             }
             __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
@@ -331,26 +327,26 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     for (int i = 0; i < 32; ++i)
                         if (cc * 32 + i >= col_limit) s[cc][i] = __float_as_uint(-INFINITY);
             }
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-                for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(s[cc][i]));
-            const float m_t = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            const float m_t = row_max128(s);
             const float m_new = fmaxf(m_run, m_t);
             const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
             const float alpha = ex2_approx((m_run - m_use) * p.c);
-            const float mc_eff = m_use * c_eff - x_bias;
             m_run = m_new;
             sScale[t * 128 + r] = alpha;
             mbar_arrive(bar_scale(t));
 
-            float l_tile = 0.f;
+            // exact: x = s*c - m*c + P offset;  h15: doubled input 2x = s*(2c) - m*(2c);  pot: x = s*c - m*c
+            RowScale rs;
+            rs.c = make_float2(c_eff, c_eff);
+            const float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
+            rs.nmc = make_float2(nmc, nmc);
+            rs.two22 = p.two22;
+            float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
             if (masked_tile) {
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     uint32_t pw[16];
-                    l_tile += weights_chunk32<FP8, MODE, true>(s[cc], c_eff, mc_eff, col_limit - cc * 32, pw);
+                    weights_chunk32<FP8, MODE, true>(s[cc], rs, col_limit - cc * 32, acc, pw);
                     if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                     else tmem_st16(tS + cc * 16, pw);
                 }
@@ -358,11 +354,12 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     uint32_t pw[16];
-                    l_tile += weights_chunk32<FP8, MODE, false>(s[cc], c_eff, mc_eff, 32, pw);
+                    weights_chunk32<FP8, MODE, false>(s[cc], rs, 32, acc, pw);
                     if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                     else tmem_st16(tS + cc * 16, pw);
                 }
             }
+            const float l_tile = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p_full(t));
@@ -383,28 +380,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 // Host launcher
 // ------------------------------------------------------------------------------------------------
 template <int D, bool FP8, int MODE>
-static cudaError_t launch_serial(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                 const AttnParams& p, cudaStream_t stream) {
-    using C = TileCfg<D, FP8>;
-    constexpr int smem_bytes = 3 * C::kTileBytes + 64 + 1024;
-    auto kern = attn_fwd_serial_kernel<D, FP8, MODE>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    dim3 grid((p.Sq + kTileM - 1) / kTileM, p.Hq, p.B);
-    kern<<<grid, 128, smem_bytes, stream>>>(tq, tk, tv, p);
-    return cudaGetLastError();
-}
-
-template <int D, bool FP8, int MODE>
 static cudaError_t launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              const AttnParams& p, cudaStream_t stream) {
     using W = WsCfg<D, FP8>;
-    static const bool serial = std::getenv("ROWMAX_ATTN_SERIAL") != nullptr;
-    if (serial) return launch_serial<D, FP8, MODE>(tq, tk, tv, p, stream);
     auto kern = attn_fwd_ws_kernel<D, FP8, MODE>;
     static bool configured = false;
     if (!configured) {
@@ -441,14 +419,15 @@ cudaError_t launch_attn_fwd(int D, bool fp8, int mode, const CUtensorMap& tq, co
 // ------------------------------------------------------------------------------------------------
 // Weight-map sweep: the same device functions on a flat array of offsets.
 // ------------------------------------------------------------------------------------------------
-__global__ void weight_map_kernel(const float* __restrict__ x, float* __restrict__ w, size_t n, int mode) {
+__global__ void weight_map_kernel(const float* __restrict__ x, float* __restrict__ w, size_t n, int mode,
+                                  uint32_t two22) {
     const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
     for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride) {
         const float xi = x[i];
         float wi;
         if (mode == kExact) wi = w_exact(xi);
         else if (mode == kPot) wi = w_pot(xi);
-        else wi = w_h15_doubled(xi * 2.0f);
+        else wi = w_h15_doubled_pair<0>(make_float2(xi * 2.0f, xi * 2.0f), two22).x;
         w[i] = wi;
     }
 }
@@ -458,7 +437,7 @@ cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cuda
     const int threads = 256;
     size_t blocks = (n + threads - 1) / threads;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    weight_map_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(x, w, n, mode);
+    weight_map_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(x, w, n, mode, 1u << 22);
     return cudaGetLastError();
 }
 

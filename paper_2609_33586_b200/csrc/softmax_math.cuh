@@ -1,4 +1,9 @@
-// Tile geometry and the per-element softmax arithmetic shared by the attention kernels.
+// Tile geometry and the per-element softmax arithmetic of the attention kernel.
+//
+// Instruction budget per score element (what the tensor cores leave for the softmax warps is about
+// 8 issue slots at bf16 and 4 at fp8, per element, at full MMA rate), so the hot loops use packed
+// two-lane fp32 instructions (fma.rn.f32x2 / add.rn.f32x2), the three-input max, and for the
+// rounding maps an integer multiply-add that builds the fp32 weight pattern on the FMA pipe.
 #pragma once
 #include "attn_kernel_common.cuh"
 #include "ptx.cuh"
@@ -19,10 +24,61 @@ struct TileCfg {
     static constexpr int kUmmaK = 32 / kElem;               // elements per MMA along K (32 bytes)
     static constexpr int kQkSteps = D / kUmmaK;
     static constexpr int kPvSteps = kTileN / kUmmaK;
-    static constexpr int kPCols = kTileN * kElem / 4;       // TMEM columns holding one P tile
     static_assert(kRowBytes % 128 == 0, "row must be a whole number of 128-byte swizzle rows");
 };
 
+// P is stored as weight * 2^kPOff so that it fills the range of its fp8 format: e4m3 holds the
+// exact-mode weights up to 2^8 = 256 <= 448; e5m2 holds the lattice weights {1, 1.5} * 2^k exactly
+// from 2^15 down to 2^-14 (k >= -29 relative to the row maximum).  The row sum carries the same
+// factor, so it cancels in O and is subtracted from LSE.
+template <bool FP8, int MODE>
+struct PFormat {
+    static constexpr int kOffLog2 = FP8 ? (MODE == kExact ? 8 : 15) : 0;
+};
+
+// ---- packed fp32 pairs and small helpers
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// (a * b + c) mod 2^32 as one integer multiply-add; b arrives in a register so that the shift it
+// stands for stays an FMA-pipe instruction.
+__device__ __forceinline__ uint32_t imad(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16_rn(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -32,62 +88,77 @@ __device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
     return r;
 }
-
-// exact-mode fp8 path stores P = w * 2^8 in e4m3 (largest value 256 <= 448)
-constexpr int kP8ExactOffsetLog2 = 8;
-
-// Turns 32 consecutive scores of one row into weights: returns their sum and writes the packed P
-// words (16 words of 2 bf16, or 8 words of 4 fp8).  `limit` = first masked column of the chunk
-// (MASKED tiles only; masked scores must already hold -inf for the exact map).
-template <bool FP8, int MODE, bool MASKED>
-__device__ __forceinline__ float weights_chunk32(const uint32_t (&sraw)[32], float c_eff, float mc_eff,
-                                                 int limit, uint32_t* pw) {
-    float acc0 = 0.f, acc1 = 0.f;
-    uint32_t pb[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const float s = __uint_as_float(sraw[i]);
-        const bool masked = MASKED && i >= limit;
-        float w;
-        uint32_t bits;  // P pattern: bf16 in the low 16 bits, or an fp8 byte
-        if constexpr (MODE == kExact) {
-            w = w_exact(fmaf(s, c_eff, -mc_eff));  // masked scores are -inf -> weight 0
-            bits = 0;
-        } else if constexpr (MODE == kH15) {
-            const uint32_t tb = h15_tbits(fmaf(s, c_eff, -mc_eff));  // c_eff = 2c: doubled input
-            w = h15_weight_from_tbits(tb);
-            bits = FP8 ? h15_e5m2_from_tbits(tb) : (__float_as_uint(w) >> 16);
-        } else {
-            const int d = pot_index(fmaf(s, c_eff, -mc_eff));
-            w = __uint_as_float(static_cast<uint32_t>(127 - d) << 23);
-            bits = FP8 ? static_cast<uint32_t>(15 + kP8OffsetLog2 - d) << 2 : (__float_as_uint(w) >> 16);
-        }
-        if constexpr (MODE != kExact && MASKED) {
-            if (masked) { w = 0.f; bits = 0; }
-        }
-        pb[i] = (MODE == kExact) ? __float_as_uint(w) : bits;
-        if (i & 1) acc1 += w; else acc0 += w;
-    }
-    if constexpr (!FP8) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            if constexpr (MODE == kExact)
-                pw[i] = pack_bf16_rn(__uint_as_float(pb[2 * i]), __uint_as_float(pb[2 * i + 1]));
-            else
-                pw[i] = pb[2 * i] | (pb[2 * i + 1] << 16);
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if constexpr (MODE == kExact)
-                pw[i] = pack_e4m3x2(__uint_as_float(pb[4 * i]), __uint_as_float(pb[4 * i + 1])) |
-                        (pack_e4m3x2(__uint_as_float(pb[4 * i + 2]), __uint_as_float(pb[4 * i + 3])) << 16);
-            else
-                pw[i] = pb[4 * i] | (pb[4 * i + 1] << 8) | (pb[4 * i + 2] << 16) | (pb[4 * i + 3] << 24);
-        }
-    }
-    return acc0 + acc1;
+__device__ __forceinline__ uint32_t pack_e5m2x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
 }
 
+// Row maximum of 128 scores held as 4 x 32 registers.
+__device__ __forceinline__ float row_max128(const uint32_t (&s)[4][32]) {
+    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+            m0 = max3(m0, __uint_as_float(s[cc][i + 0]), __uint_as_float(s[cc][i + 1]));
+            m1 = max3(m1, __uint_as_float(s[cc][i + 2]), __uint_as_float(s[cc][i + 3]));
+            m2 = max3(m2, __uint_as_float(s[cc][i + 4]), __uint_as_float(s[cc][i + 5]));
+            m3 = max3(m3, __uint_as_float(s[cc][i + 6]), __uint_as_float(s[cc][i + 7]));
+        }
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// Per-row constants of the weight map for one key tile.
+struct RowScale {
+    float2 c;      // multiplier of the raw score (c, or 2c for the doubled h15 input), both lanes
+    float2 nmc;    // minus the scaled anchor (plus the P offset in exact mode), both lanes
+    uint32_t two22;  // 1 << 22 held in a register (see imad)
+};
+
+// Turns 32 consecutive scores of one row into weights.  Adds them (times 2^kOffLog2) into `acc`
+// (two independent packed accumulators, summed by the caller)
+// and writes the packed P words: 16 words of 2 bf16, or 8 words of 4 fp8.  In a MASKED tile
+// columns >= limit are masked: their scores already hold -inf and their weights are forced to 0.
+template <bool FP8, int MODE, bool MASKED>
+__device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const RowScale& rs, int limit,
+                                                float2 (&acc)[2], uint32_t* pw) {
+    constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
+    uint32_t half16[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float2 sv = make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+        float2 x = ffma2(sv, rs.c, rs.nmc);
+        float2 w;
+        if constexpr (MODE == kExact) {
+            w.x = w_exact(x.x);  // masked scores are -inf -> weight 0
+            w.y = w_exact(x.y);
+        } else if constexpr (MODE == kH15) {
+            // Eq. h15 on the doubled input: clamp at -252, add 2^23 + 2^22 (rounds to the integer n,
+            // ties to even), then (bits << 22) + bias builds (1 + (n mod 2)/2) * 2^(floor(n/2) + kOff).
+            w = w_h15_doubled_pair<kOff>(x, rs.two22);
+        } else {
+            w.x = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.x)) << 23);
+            w.y = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.y)) << 23);
+        }
+        if constexpr (MODE != kExact && MASKED) {
+            if (2 * i >= limit) w.x = 0.f;
+            if (2 * i + 1 >= limit) w.y = 0.f;
+        }
+        acc[i & 1] = fadd2(acc[i & 1], w);
+        if constexpr (!FP8) {
+            if constexpr (MODE == kExact) pw[i] = pack_bf16_rn(w.x, w.y);
+            else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: 1 fraction bit
+        } else {
+            if constexpr (MODE == kExact) half16[i] = pack_e4m3x2(w.x, w.y);
+            else half16[i] = pack_e5m2x2(w.x, w.y);  // exact wherever e5m2 can hold the weight
+        }
+    }
+    if constexpr (FP8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pw[i] = __byte_perm(half16[2 * i], half16[2 * i + 1], 0x5410);
+    }
+}
 
 }  // namespace rowmax

@@ -30,17 +30,26 @@ __device__ __forceinline__ float h15_weight_from_tbits(uint32_t tbits) {
     return __uint_as_float((tbits << 22) + 0x3F800000u);
 }
 __device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_from_tbits(h15_tbits(x2)); }
-// bf16 pattern of the same weight: the upper half of the fp32 pattern, (n + 254) << 6.  Exact.
-__device__ __forceinline__ uint32_t h15_bf16_from_tbits(uint32_t tbits) {
-    return ((tbits << 22) + 0x3F800000u) >> 16;
-}
-// e5m2 pattern of weight * 2^15: exponent field floor(n/2) + 30, top fraction bit n mod 2, i.e.
-// (n + 60) << 1.  Exact for n >= -58; below that the stored P flushes toward zero (relative to the
-// row maximum this is under 2^-29; the row sum still uses the fp32 weight).
-constexpr int kP8OffsetLog2 = 15;
-__device__ __forceinline__ uint32_t h15_e5m2_from_tbits(uint32_t tbits) {
-    int n60 = static_cast<int>(tbits - kH15MagicBits) + 4 * kP8OffsetLog2;
-    return static_cast<uint32_t>(max(n60, 0)) << 1;
+// Two weights at once, the form the fused kernel uses: packed fp32 add of the magic constant, then
+// one integer multiply-add per lane, t * 2^22 + bias (mod 2^32), equal to (bits << 22) + bias.
+// `two22` must hold 1 << 22; it is passed in a register so that the multiply-add stays on the FMA
+// pipe.  kOff scales the weight by 2^kOff (an exact exponent shift) for the fp8 P formats.
+template <int kOff>
+__device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) {
+    x2.x = fmaxf(x2.x, -252.0f);
+    x2.y = fmaxf(x2.y, -252.0f);
+    float2 t;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(t.x), "=f"(t.y)
+        : "f"(x2.x), "f"(x2.y), "f"(kH15Magic));
+    constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(2 * kOff) << 22);
+    uint32_t b0, b1;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b0) : "r"(__float_as_uint(t.x)), "r"(two22), "r"(bias));
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22), "r"(bias));
+    return make_float2(__uint_as_float(b0), __uint_as_float(b1));
 }
 
 // ---- Rowmax-PoT (Eq. rowmax-pot): d = min{K_max, floor(y + 1/2)}, y = -x, w = 2^-d.
