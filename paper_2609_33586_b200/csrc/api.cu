@@ -19,6 +19,10 @@ cudaError_t status_word_address(int** out);
 namespace {
 
 std::atomic<unsigned long long> g_launches{0};
+#ifdef ROWMAX_TRACE
+long long* g_trace = nullptr;
+int g_trace_block = 0;
+#endif
 int g_last_cuda_error = 0;
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -100,6 +104,14 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 extern "C" {
 
+#ifdef ROWMAX_TRACE
+// Trace builds only: device buffer of 4 * 64 * 8 int64 that CTA `block` fills with cycle stamps.
+void attn_set_trace(long long* device_buffer, int block) {
+    g_trace = device_buffer;
+    g_trace_block = block;
+}
+#endif
+
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
              int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
              float k_descale, float v_descale, void* stream) {
@@ -131,6 +143,10 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
     p.c = static_cast<float>(static_cast<double>(softmax_scale) * dq * dk * 1.4426950408889634074);
     p.v_descale = fp8 ? v_descale : 1.0f;
     p.two22 = 1u << 22;
+#ifdef ROWMAX_TRACE
+    p.trace = g_trace;
+    p.trace_block = g_trace_block;
+#endif
     rc = status_word(&p.status);
     if (rc != ATTN_OK) return rc;
 

@@ -42,6 +42,18 @@ __device__ __forceinline__ void reg_dec_48() { asm volatile("setmaxnreg.dec.sync
 __device__ __forceinline__ void reg_dec_80() { asm volatile("setmaxnreg.dec.sync.aligned.u32 80;"); }
 __device__ __forceinline__ void reg_inc_192() { asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); }
 
+// Optional cycle stamps (compiled in only with -DROWMAX_TRACE): one representative thread per role of
+// one chosen CTA writes clock64() at fixed points of its first 64 key tiles.
+#ifdef ROWMAX_TRACE
+#define ROWMAX_STAMP(role, j, slot)                                                              \
+    do {                                                                                         \
+        if (p.trace != nullptr && static_cast<int>(blockIdx.x) == p.trace_block && (j) < 64)     \
+            p.trace[((role) * 64 + (j)) * 8 + (slot)] = clock64();                               \
+    } while (0)
+#else
+#define ROWMAX_STAMP(role, j, slot) do { } while (0)
+#endif
+
 enum BarId : int { kBarQ = 0, kBarKvFull = 1, kBarKvEmpty = 2, kBarSFull = 3, kBarPFull = 4, kBarOFull = 5,
                    kBarScale = 6, kBarORescaled = 7, kBarFinal = 8 };
 
@@ -154,25 +166,33 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     }
                 }
             }
-        } else if (warp == 12 && lane == 0) {
+        } else if (warp == 12) {
             // ------------------------------------------------------------ MMA issuer
-            auto issue_s = [&](int t, uint32_t sK) {
-                const uint32_t q = sQ + t * C::kTileBytes;
+            // The whole warp walks the loop (so addresses and descriptors stay warp-uniform values);
+            // one elected lane issues the MMAs and commits.
+            const bool leader = elect_one();
+            constexpr uint32_t desc_hi = umma_desc_hi_sw128(1024);
+            const uint32_t q_lo0 = umma_desc_lo(sQ, 16);
+            const uint32_t ring_lo_k = umma_desc_lo(sRing, 16);               // K tiles: K-major
+            const uint32_t ring_lo_v = umma_desc_lo(sRing, C::kBoxBytes);     // V tiles: MN-major, LBO = next 128-byte column block
+            constexpr uint32_t kTileLo = C::kTileBytes >> 4;
+            auto issue_s = [&](int t, uint32_t k_lo) {
+                const uint32_t q_lo = q_lo0 + t * kTileLo;
 #pragma unroll
                 for (int ks = 0; ks < C::kQkSteps; ++ks) {
-                    const uint32_t off = (ks / 4) * C::kBoxBytes + (ks % 4) * 32;
-                    umma_ss<FP8>(tmem_S(t), umma_desc_sw128(q + off, 16, 1024), umma_desc_sw128(sK + off, 16, 1024),
-                                 idesc_s, ks > 0);
+                    const uint32_t off = ((ks / 4) * C::kBoxBytes + (ks % 4) * 32) >> 4;
+                    umma_ss_lo<FP8>(tmem_S(t), q_lo + off, k_lo + off, desc_hi, idesc_s, ks > 0 ? 1u : 0u);
                 }
             };
-            auto issue_pv = [&](int t, uint32_t sV, bool accumulate) {
+            auto issue_pv = [&](int t, uint32_t v_lo, bool accumulate) {
 #pragma unroll
                 for (int ks = 0; ks < C::kPvSteps; ++ks) {
-                    const uint64_t bdesc = umma_desc_sw128(sV + ks * C::kUmmaK * 128, C::kBoxBytes, 1024);
-                    umma_ts<FP8>(tmem_O(t), tmem_S(t) + ks * 8, bdesc, idesc_pv, (accumulate || ks > 0) ? 1u : 0u);
+                    const uint32_t off = (ks * C::kUmmaK * 128) >> 4;
+                    umma_ts_lo<FP8>(tmem_O(t), tmem_S(t) + ks * 8, v_lo + off, desc_hi, idesc_pv,
+                                    (accumulate || ks > 0) ? 1u : 0u);
                 }
             };
-            auto slot_addr = [&](int idx) { return sRing + (idx % NS) * C::kTileBytes; };
+            auto slot_lo = [&](int idx) { return static_cast<uint32_t>(idx % NS) * kTileLo; };
             auto wait_full = [&](int idx) {
                 mbar_wait(bar_kv_full(idx % NS), (idx / NS) & 1, wctx, (kRoleMma << 8) | kBarKvFull);
             };
@@ -183,11 +203,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     if (n_t[t] > 0) {
                         mbar_wait(bar_q(t), 0, wctx, (kRoleMma << 8) | kBarQ);
                         tc_fence_after();
-                        if (!*abort_flag) issue_s(t, slot_addr(0));
-                        umma_commit(bar_s_full(t));
+                        if (leader) {
+                            if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(0));
+                            umma_commit(bar_s_full(t));
+                        }
                     }
                 }
-                umma_commit(bar_kv_empty(0));
+                if (leader) umma_commit(bar_kv_empty(0));
                 for (int j = 0; j < n_max; ++j) {
                     wait_full(2 * j + 1);
                     bool k_ready = false;
@@ -195,10 +217,15 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     for (int t = 0; t < 2; ++t) {
                         if (j < n_t[t]) {
                             mbar_wait(bar_p_full(t), j & 1, wctx, (kRoleMma << 8) | kBarPFull);
+                            if (leader) ROWMAX_STAMP(3, j, t * 4 + 0);
                             mbar_wait(bar_o_rescaled(t), j & 1, wctx, (kRoleMma << 8) | kBarORescaled);
+                            if (leader) ROWMAX_STAMP(3, j, t * 4 + 1);
                             tc_fence_after();
-                            if (!*abort_flag) issue_pv(t, slot_addr(2 * j + 1), j > 0);
-                            umma_commit(bar_o_full(t));
+                            if (leader) {
+                                if (!*abort_flag) issue_pv(t, ring_lo_v + slot_lo(2 * j + 1), j > 0);
+                                umma_commit(bar_o_full(t));
+                                ROWMAX_STAMP(3, j, t * 4 + 2);
+                            }
                         }
                         if (j + 1 < n_t[t]) {
                             if (!k_ready) {
@@ -206,12 +233,18 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                                 tc_fence_after();
                                 k_ready = true;
                             }
-                            if (!*abort_flag) issue_s(t, slot_addr(2 * j + 2));
-                            umma_commit(bar_s_full(t));
+                            if (leader) {
+                                if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(2 * j + 2));
+                                umma_commit(bar_s_full(t));
+                                ROWMAX_STAMP(3, j, t * 4 + 3);
+                            }
                         }
                     }
-                    umma_commit(bar_kv_empty((2 * j + 1) % NS));
-                    if (j + 1 < n_max) umma_commit(bar_kv_empty((2 * j + 2) % NS));
+                    if (leader) {
+                        umma_commit(bar_kv_empty((2 * j + 1) % NS));
+                        if (j + 1 < n_max) umma_commit(bar_kv_empty((2 * j + 2) % NS));
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -225,9 +258,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             for (int t = 0; t < 2; ++t) {
                 if (j < n_t[t]) {
                     mbar_wait(bar_scale(t), j & 1, wctx, (kRoleCorr << 8) | kBarScale);
+                    if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 0);
                     const float alpha = sScale[t * 128 + r];
                     if (j > 0) {
                         mbar_wait(bar_o_full(t), (j - 1) & 1, wctx, (kRoleCorr << 8) | kBarOFull);
+                        if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 1);
                         __syncwarp();
                         tc_fence_after();
                         if (__any_sync(0xffffffffu, alpha != 1.0f)) {
@@ -237,7 +272,12 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                                 tmem_ld32(tmem_O(t) + lane_base + cc * 32, o);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                for (int i = 0; i < 32; i += 2) {
+                                    const float2 v = fmul2(make_float2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])),
+                                                           make_float2(alpha, alpha));
+                                    o[i] = __float_as_uint(v.x);
+                                    o[i + 1] = __float_as_uint(v.y);
+                                }
                                 tmem_st32(tmem_O(t) + lane_base + cc * 32, o);
                             }
                             tmem_wait_st();
@@ -245,6 +285,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         tc_fence_before();
                     }
                     mbar_arrive(bar_o_rescaled(t));
+                    if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 2);
                 }
             }
         }
@@ -311,12 +352,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         float m_run = -INFINITY, l_run = 0.f;
         for (int j = 0; j < nt; ++j) {
             mbar_wait(bar_s_full(t), j & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);
+            if (r == 0) ROWMAX_STAMP(t, j, 0);
             __syncwarp();
             tc_fence_after();
             uint32_t s[4][32];
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, s[cc]);
             tmem_wait_ld();
+            if (r == 0) ROWMAX_STAMP(t, j, 1);
 
             const bool masked_tile = (j + 1) * kTileN > tile_limit;
             const int col_limit = row_limit - j * kTileN;
@@ -334,6 +377,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             m_run = m_new;
             sScale[t * 128 + r] = alpha;
             mbar_arrive(bar_scale(t));
+            if (r == 0) ROWMAX_STAMP(t, j, 2);
 
             // exact: x = s*c - m*c + P offset;  h15: doubled input 2x = s*(2c) - m*(2c);  pot: x = s*c - m*c
             RowScale rs;
@@ -360,9 +404,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 }
             }
             const float l_tile = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
+            if (r == 0) ROWMAX_STAMP(t, j, 3);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p_full(t));
+            if (r == 0) ROWMAX_STAMP(t, j, 4);
             l_run = l_run * alpha + l_tile;
         }
         if (nt > 0) {

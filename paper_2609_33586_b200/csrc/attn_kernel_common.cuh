@@ -20,6 +20,10 @@ struct AttnParams {
     float v_descale;  // 1 for bf16
     uint32_t two22;   // 1 << 22, kept in a register for the h15 integer multiply-add
     int* status;      // device-global sticky status word
+#ifdef ROWMAX_TRACE
+    long long* trace;  // optional per-role cycle stamps of one CTA: [role 4][tile 64][slot 8]
+    int trace_block;
+#endif
 };
 
 // Status codes written by expired waits: role << 8 | barrier id.
