@@ -32,7 +32,7 @@ struct WsCfg {
     static constexpr int kScaleOff = kQBytes + kRingBytes;        // float alpha[2][128]
     static constexpr int kFinalOff = kScaleOff + 2 * 128 * 4;     // float2 (l, m)[2][128]
     static constexpr int kBarOff = kFinalOff + 2 * 128 * 8;
-    static constexpr int kNumBars = 2 + 2 * kSlots + 6 * 2;
+    static constexpr int kNumBars = 2 + 2 * kSlots + 6 * 2 + 8;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kSmemBytes = kMiscOff + 16 + 1024;       // + manual 1024-byte alignment slack
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
@@ -54,8 +54,12 @@ __device__ __forceinline__ void reg_inc_192() { asm volatile("setmaxnreg.inc.syn
 #define ROWMAX_STAMP(role, j, slot) do { } while (0)
 #endif
 
+// Whether the two softmax warps of a scheduler alternate strictly (see the softmax role).  Measured
+// slower than free-running on every workload tried, so it is off; the barriers stay for experiments.
+constexpr bool kTakeTurns = false;
+
 enum BarId : int { kBarQ = 0, kBarKvFull = 1, kBarKvEmpty = 2, kBarSFull = 3, kBarPFull = 4, kBarOFull = 5,
-                   kBarScale = 6, kBarORescaled = 7, kBarFinal = 8 };
+                   kBarScale = 6, kBarORescaled = 7, kBarFinal = 8, kBarTurn = 9 };
 
 }  // namespace
 
@@ -88,6 +92,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto bar_scale = [&](int t) { return bar_x(3, t); };       // softmax -> correction: alpha_t(j) in smem
     auto bar_o_rescaled = [&](int t) { return bar_x(4, t); };  // correction -> MMA: O_t rescaled for tile j
     auto bar_final = [&](int t) { return bar_x(5, t); };       // softmax -> correction: (l, m) in smem
+    // turn token of the softmax warp pair that shares scheduler w: bar_turn(t, w) lets tile t's warp go
+    auto bar_turn = [&](int t, int w) { return bar0 + 8u * (2 + 2 * NS + 12 + 4 * t + w); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
 
@@ -121,6 +127,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             mbar_init(bar_scale(t), 128);
             mbar_init(bar_o_rescaled(t), 128);
             mbar_init(bar_final(t), 128);
+            for (int w = 0; w < 4; ++w) mbar_init(bar_turn(t, w), 1);
         }
         *abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0);
         fence_mbar_init();
@@ -344,6 +351,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t tS = tmem_S(t) + lane_base;
         const int q0 = t == 0 ? q0t[0] : q0t[1];
         const int nt = t == 0 ? n_t[0] : n_t[1];
+        // The two softmax warps on one scheduler take turns on their arithmetic-heavy section, tile by
+        // tile (0, 1, 0, 1, ...), so that each runs it alone and the two query tiles stay half a period
+        // apart: while one warp computes weights, the other's MMAs and hand-offs are in flight.
+        const int n_both = kTakeTurns ? min(n_t[0], n_t[1]) : 0;   // tiles for which both warps are active
+        const int w4 = warp & 3;
         const int row = q0 + r;
         const int row_limit = p.causal ? min(p.Sk, row + shift + 1) : p.Sk;  // visible keys of this row
         // first key index that some row of this tile cannot see (tile-uniform)
@@ -352,6 +364,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         float m_run = -INFINITY, l_run = 0.f;
         for (int j = 0; j < nt; ++j) {
             mbar_wait(bar_s_full(t), j & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);
+            if (t == 0) {
+                if (j > 0 && j < n_both) mbar_wait(bar_turn(0, w4), (j - 1) & 1, wctx, (kRoleSoftmax << 8) | kBarTurn);
+            } else {
+                if (j < n_both) mbar_wait(bar_turn(1, w4), j & 1, wctx, (kRoleSoftmax << 8) | kBarTurn);
+            }
             if (r == 0) ROWMAX_STAMP(t, j, 0);
             __syncwarp();
             tc_fence_after();
@@ -405,6 +422,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             const float l_tile = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
             if (r == 0) ROWMAX_STAMP(t, j, 3);
+            __syncwarp();
+            if (lane == 0) {   // pass the turn to the other tile's warp
+                if (t == 0) {
+                    if (j < n_both) mbar_arrive(bar_turn(1, w4));
+                } else {
+                    if (j + 1 < n_both) mbar_arrive(bar_turn(0, w4));
+                }
+            }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p_full(t));

@@ -88,26 +88,27 @@ __device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
     return r;
 }
-__device__ __forceinline__ uint32_t pack_e5m2x2(float lo, float hi) {
-    uint16_t r;
-    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+__device__ __forceinline__ uint32_t pack_f16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
 
 // Row maximum of 128 scores held as 4 x 32 registers.
 __device__ __forceinline__ float row_max128(const uint32_t (&s)[4][32]) {
-    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+    float m[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) m[a] = -INFINITY;
 #pragma unroll
     for (int cc = 0; cc < 4; ++cc) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-            m0 = max3(m0, __uint_as_float(s[cc][i + 0]), __uint_as_float(s[cc][i + 1]));
-            m1 = max3(m1, __uint_as_float(s[cc][i + 2]), __uint_as_float(s[cc][i + 3]));
-            m2 = max3(m2, __uint_as_float(s[cc][i + 4]), __uint_as_float(s[cc][i + 5]));
-            m3 = max3(m3, __uint_as_float(s[cc][i + 6]), __uint_as_float(s[cc][i + 7]));
+        for (int i = 0; i < 32; i += 16) {
+#pragma unroll
+            for (int a = 0; a < 8; ++a)
+                m[a] = max3(m[a], __uint_as_float(s[cc][i + 2 * a]), __uint_as_float(s[cc][i + 2 * a + 1]));
         }
     }
-    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+    return fmaxf(max3(m[0], m[1], m[2]), max3(m[3], m[4], max3(m[5], m[6], m[7])));
 }
 
 // Per-row constants of the weight map for one key tile.
@@ -152,12 +153,15 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: 1 fraction bit
         } else {
             if constexpr (MODE == kExact) half16[i] = pack_e4m3x2(w.x, w.y);
-            else half16[i] = pack_e5m2x2(w.x, w.y);  // exact wherever e5m2 can hold the weight
+            else half16[i] = pack_f16x2_rn(w.x, w.y);  // lattice weights are exact in fp16 (1 fraction bit)
         }
     }
     if constexpr (FP8) {
+        // exact mode: two e4m3 pairs per word.  pot/h15: e5m2 is the upper byte of an fp16 pattern, and a
+        // lattice weight has one fraction bit, so the upper bytes of the four halves are the exact P bytes.
 #pragma unroll
-        for (int i = 0; i < 8; ++i) pw[i] = __byte_perm(half16[2 * i], half16[2 * i + 1], 0x5410);
+        for (int i = 0; i < 8; ++i)
+            pw[i] = __byte_perm(half16[2 * i], half16[2 * i + 1], MODE == kExact ? 0x5410 : 0x7531);
     }
 }
 

@@ -46,9 +46,9 @@ __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) 
         : "=f"(t.x), "=f"(t.y)
         : "f"(x2.x), "f"(x2.y), "f"(kH15Magic));
     constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(2 * kOff) << 22);
-    uint32_t b0, b1;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b0) : "r"(__float_as_uint(t.x)), "r"(two22), "r"(bias));
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22), "r"(bias));
+    (void)two22;
+    const uint32_t b0 = (__float_as_uint(t.x) << 22) + bias;
+    const uint32_t b1 = (__float_as_uint(t.y) << 22) + bias;
     return make_float2(__uint_as_float(b0), __uint_as_float(b1));
 }
 
