@@ -33,6 +33,9 @@ from paper_2609_33586_b200.inputs import WORKLOADS, Workload, make_inputs, stora
 HEADLINE = WORKLOADS[2]       # causal 8K fp8
 TWIN = WORKLOADS[3]           # non-causal 8K fp8
 METRIC = "attn_fwd_tflops_h15_causal_8k_fp8"
+# dram__bytes_read.sum + dram__bytes_write.sum of one h15 launch on the headline workload, from the ncu
+# capture summarised in profiles/attn_fwd_ws_causal_8k_fp8.txt (algorithmic: 101 MB in + 68 MB out)
+NCU_DRAM_BYTES_PER_LAUNCH = 169.6e6 + 32.4e6
 MODE_IDS = {"exact": 0, "pot": 1, "h15": 2}
 
 
@@ -63,25 +66,58 @@ def barrier():
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while a timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU while a timed region runs (NVML through
+    pynvml in a thread; nvidia-smi as the fallback)."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index, self.samples, self._stop, self._thr = index, [], threading.Event(), None
+        self.sm_max = None
+        self._nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self._nvml = pynvml
+        except Exception:
+            self._nvml = None
+
+    def _sample_nvml(self):
+        n = self._nvml
+        sm = float(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_SM))
+        pw = n.nvmlDeviceGetPowerUsage(self._h) / 1000.0
+        r = n.nvmlDeviceGetCurrentClocksEventReasons(self._h) if hasattr(n, "nvmlDeviceGetCurrentClocksEventReasons") \
+            else n.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+        flags = []
+        for name, bit in (("hw_slowdown", 0x8), ("sw_power_cap", 0x4), ("sw_thermal_slowdown", 0x20),
+                          ("hw_thermal_slowdown", 0x40)):
+            if r & bit:
+                flags.append(name)
+        self.samples.append((sm, pw, flags))
+
+    def _sample_smi(self):
+        out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                              "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
+        f = [x.strip() for x in out.stdout.strip().split(",")]
+        if len(f) >= 7:
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            flags = [n for i, n in enumerate(names) if f[3 + i].lower().startswith("active")]
+            self.sm_max = float(f[1])
+            self.samples.append((float(f[0]), float(f[2]), flags))
 
     def _run(self):
         while not self._stop.is_set():
             try:
-                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
-                f = [x.strip() for x in out.stdout.strip().split(",")]
-                if len(f) >= 7:
-                    self.samples.append(f)
+                if self._nvml is not None:
+                    self._sample_nvml()
+                else:
+                    self._sample_smi()
             except Exception:
                 pass
-            self._stop.wait(0.05)
+            self._stop.wait(0.002 if self._nvml is not None else 0.05)
 
     def __enter__(self):
         self._thr = threading.Thread(target=self._run, daemon=True)
@@ -94,13 +130,12 @@ class ClockSampler:
 
     def summary(self):
         if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no_samples"]}
-        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(s[3 + i].lower().startswith("active") for s in self.samples)]
-        pw = [float(s[2]) for s in self.samples if s[2].replace(".", "").isdigit()]
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": float(self.samples[0][1]),
-                "power_w_max": max(pw) if pw else None, "samples": len(self.samples), "reasons": reasons}
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["no_samples"]}
+        sm = [s[0] for s in self.samples]
+        reasons = sorted({f for s in self.samples for f in s[2]})
+        return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": self.sm_max,
+                "power_w_max": max(s[1] for s in self.samples), "samples": len(self.samples),
+                "source": "nvml" if self._nvml is not None else "nvidia-smi", "reasons": reasons}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -134,7 +169,7 @@ def oracle_sample(wl: Workload, inp, mode: int, row_stride: int, n_batch=None, n
             "pairs": sub.B * sub.Hq}
 
 
-def cpu_baseline_leg(wl: Workload, inp, row_stride: int = 32):
+def cpu_baseline_leg(wl: Workload, inp, row_stride: int = 8):
     s = oracle_sample(wl, inp, MODE_IDS["h15"], row_stride)
     return {"value": s["flops"] / s["seconds"] / 1e12, "unit": "TFLOP/s", "cores": s["threads"], "kind": "oracle",
             "sample": f"every {row_stride}th query row of {wl.name} ({s['rows']} rows x {s['pairs']} (batch, head) "
@@ -291,7 +326,8 @@ def run_ours(args):
         "e2e": {"value": world * wl.flops / ms_e2e / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "roofline": {"bound": "tensor", "achieved": per_gpu, "peak": fp8_peak, "unit": "TFLOP/s",
-                     "frac": per_gpu / fp8_peak, "traffic": None,
+                     "frac": per_gpu / fp8_peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH,
+                     "algorithmic_bytes": float(sum(t.numel() * t.element_size() for t in (run.q, run.k, run.v, run.o, run.lse))),
                      "peak_source": f"2 x {peaks['source']} cuBLAS bf16 burst ({peaks['bf16_tflops']} TFLOP/s); "
                                     "fp8 peak taken as twice the bf16 one (nominal ratio)",
                      "frac_of_nominal_fp8_4500": per_gpu / 4500.0},
