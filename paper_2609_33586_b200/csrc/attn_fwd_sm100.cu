@@ -57,6 +57,7 @@ __device__ __forceinline__ void reg_inc_192() { asm volatile("setmaxnreg.inc.syn
 // Whether the two softmax warps of a scheduler alternate strictly (see the softmax role).  Measured
 // slower than free-running on every workload tried, so it is off; the barriers stay for experiments.
 constexpr bool kTakeTurns = false;
+constexpr bool kStagger = true;
 
 enum BarId : int { kBarQ = 0, kBarKvFull = 1, kBarKvEmpty = 2, kBarSFull = 3, kBarPFull = 4, kBarOFull = 5,
                    kBarScale = 6, kBarORescaled = 7, kBarFinal = 8, kBarTurn = 9 };
@@ -122,11 +123,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar_s_full(t), 1);
-            mbar_init(bar_p_full(t), 128);
+            mbar_init(bar_p_full(t), 4);      // one arrival per softmax warp
             mbar_init(bar_o_full(t), 1);
-            mbar_init(bar_scale(t), 128);
-            mbar_init(bar_o_rescaled(t), 128);
-            mbar_init(bar_final(t), 128);
+            mbar_init(bar_scale(t), 4);
+            mbar_init(bar_o_rescaled(t), 4);  // one arrival per correction warp
+            mbar_init(bar_final(t), 4);
             for (int w = 0; w < 4; ++w) mbar_init(bar_turn(t, w), 1);
         }
         *abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0);
@@ -209,6 +210,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 for (int t = 0; t < 2; ++t) {
                     if (n_t[t] > 0) {
                         mbar_wait(bar_q(t), 0, wctx, (kRoleMma << 8) | kBarQ);
+                        // Stagger the two query tiles: tile 1 starts once tile 0's first P is done, which
+                        // spreads the two tiles' softmax phases apart for the first iterations.
+                        if (kStagger && t == 1 && n_t[0] > 0)
+                            mbar_wait(bar_p_full(0), 0, wctx, (kRoleMma << 8) | kBarPFull);
                         tc_fence_after();
                         if (leader) {
                             if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(0));
@@ -291,7 +296,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         }
                         tc_fence_before();
                     }
-                    mbar_arrive(bar_o_rescaled(t));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_o_rescaled(t));
                     if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 2);
                 }
             }
@@ -393,7 +399,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const float alpha = ex2_approx((m_run - m_use) * p.c);
             m_run = m_new;
             sScale[t * 128 + r] = alpha;
-            mbar_arrive(bar_scale(t));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_scale(t));
             if (r == 0) ROWMAX_STAMP(t, j, 2);
 
             // exact: x = s*c - m*c + P offset;  h15: doubled input 2x = s*(2c) - m*(2c);  pot: x = s*c - m*c
@@ -412,12 +419,30 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     else tmem_st16(tS + cc * 16, pw);
                 }
             } else {
+                // h15: the clamp at -252 is a no-op unless some score of the warp's rows lies more than
+                // 126 octaves below its running maximum; the row minimum (one more three-input pass)
+                // tells, and the common case runs without the per-score clamp.
+                bool clamp = false;
+                if constexpr (MODE == kH15) {
+                    const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest doubled offset of the row
+                    clamp = __any_sync(0xffffffffu, !(lowest >= -250.0f));
+                }
+                if (clamp) {
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t pw[16];
-                    weights_chunk32<FP8, MODE, false>(s[cc], rs, 32, acc, pw);
-                    if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
-                    else tmem_st16(tS + cc * 16, pw);
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pw[16];
+                        weights_chunk32<FP8, MODE, false, true>(s[cc], rs, 32, acc, pw);
+                        if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
+                        else tmem_st16(tS + cc * 16, pw);
+                    }
+                } else {
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pw[16];
+                        weights_chunk32<FP8, MODE, false, false>(s[cc], rs, 32, acc, pw);
+                        if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
+                        else tmem_st16(tS + cc * 16, pw);
+                    }
                 }
             }
             const float l_tile = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
@@ -432,13 +457,15 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_p_full(t));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p_full(t));
             if (r == 0) ROWMAX_STAMP(t, j, 4);
             l_run = l_run * alpha + l_tile;
         }
         if (nt > 0) {
             sFinal[t * 128 + r] = make_float2(l_run, m_run);
-            mbar_arrive(bar_final(t));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_final(t));
         }
     }
 

@@ -111,6 +111,28 @@ __device__ __forceinline__ float row_max128(const uint32_t (&s)[4][32]) {
     return fmaxf(max3(m[0], m[1], m[2]), max3(m[3], m[4], max3(m[5], m[6], m[7])));
 }
 
+// Row minimum of the same 128 scores (decides whether the h15 clamp can be skipped for a tile).
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float row_min128(const uint32_t (&s)[4][32]) {
+    float m[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) m[a] = INFINITY;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 16) {
+#pragma unroll
+            for (int a = 0; a < 8; ++a)
+                m[a] = min3(m[a], __uint_as_float(s[cc][i + 2 * a]), __uint_as_float(s[cc][i + 2 * a + 1]));
+        }
+    }
+    return fminf(min3(m[0], m[1], m[2]), min3(m[3], m[4], min3(m[5], m[6], m[7])));
+}
+
 // Per-row constants of the weight map for one key tile.
 struct RowScale {
     float2 c;      // multiplier of the raw score (c, or 2c for the doubled h15 input), both lanes
@@ -122,7 +144,8 @@ struct RowScale {
 // (two independent packed accumulators, summed by the caller)
 // and writes the packed P words: 16 words of 2 bf16, or 8 words of 4 fp8.  In a MASKED tile
 // columns >= limit are masked: their scores already hold -inf and their weights are forced to 0.
-template <bool FP8, int MODE, bool MASKED>
+// CLAMP = false (h15 only) may be used when every doubled offset of the chunk is known to be >= -252.
+template <bool FP8, int MODE, bool MASKED, bool CLAMP = true>
 __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const RowScale& rs, int limit,
                                                 float2 (&acc)[2], uint32_t* pw) {
     constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
@@ -138,7 +161,7 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
         } else if constexpr (MODE == kH15) {
             // Eq. h15 on the doubled input: clamp at -252, add 2^23 + 2^22 (rounds to the integer n,
             // ties to even), then (bits << 22) + bias builds (1 + (n mod 2)/2) * 2^(floor(n/2) + kOff).
-            w = w_h15_doubled_pair<kOff>(x, rs.two22);
+            w = w_h15_doubled_pair<kOff, CLAMP>(x, rs.two22);
         } else {
             w.x = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.x)) << 23);
             w.y = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.y)) << 23);

@@ -31,13 +31,17 @@ __device__ __forceinline__ float h15_weight_from_tbits(uint32_t tbits) {
 }
 __device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_from_tbits(h15_tbits(x2)); }
 // Two weights at once, the form the fused kernel uses: packed fp32 add of the magic constant, then
-// one integer multiply-add per lane, t * 2^22 + bias (mod 2^32), equal to (bits << 22) + bias.
-// `two22` must hold 1 << 22; it is passed in a register so that the multiply-add stays on the FMA
-// pipe.  kOff scales the weight by 2^kOff (an exact exponent shift) for the fp8 P formats.
-template <int kOff>
+// (bits << 22) + bias per lane.  One lane uses the shift-add (ALU pipe), the other the equivalent
+// integer multiply-add t * 2^22 + bias mod 2^32 (FMA pipe), which balances the two pipes; `two22`
+// must hold 1 << 22 and arrives in a register so that the multiply-add is not turned back into a
+// shift.  kOff scales the weight by 2^kOff (an exact exponent shift) for the fp8 P formats.
+// kClamp = false skips the clamp at -252; the caller must know that both inputs are >= -252.
+template <int kOff, bool kClamp = true>
 __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) {
-    x2.x = fmaxf(x2.x, -252.0f);
-    x2.y = fmaxf(x2.y, -252.0f);
+    if constexpr (kClamp) {
+        x2.x = fmaxf(x2.x, -252.0f);
+        x2.y = fmaxf(x2.y, -252.0f);
+    }
     float2 t;
     asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
         "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
@@ -46,9 +50,9 @@ __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) 
         : "=f"(t.x), "=f"(t.y)
         : "f"(x2.x), "f"(x2.y), "f"(kH15Magic));
     constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(2 * kOff) << 22);
-    (void)two22;
     const uint32_t b0 = (__float_as_uint(t.x) << 22) + bias;
-    const uint32_t b1 = (__float_as_uint(t.y) << 22) + bias;
+    uint32_t b1;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22), "r"(bias));
     return make_float2(__uint_as_float(b0), __uint_as_float(b1));
 }
 

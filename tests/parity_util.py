@@ -41,8 +41,13 @@ def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None):
                     tie_eps=TIE_EPS if mode != orc.W_EXACT else 0.0, rows=rows)
 
 
-def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, device="cuda:0"):
-    """Returns a dict of error statistics; `ok` says whether every gate holds."""
+def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, device="cuda:0",
+            allow_output_rounding: bool = False):
+    """Returns a dict of error statistics; `ok` says whether every gate holds.
+
+    `allow_output_rounding` adds half a bf16 ulp of the reference value to the per-row tolerance: O
+    is stored in bf16, and for outputs of magnitude 2 and above that rounding alone is 0.008 and
+    more.  The standard workloads (N(0,1) values, averaged) do not need it."""
     inp = inp or make_inputs(wl)
     o, lse = run_cuda(wl, inp, mode, device)
     ref = run_oracle(wl, inp, mode, rows)
@@ -53,8 +58,9 @@ def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, devic
     tol = TOL[wl.in_dtype]
     err_o = np.abs(o - ref["O"])
     row_err = err_o.max(axis=-1)
-    # bf16 rounding of the stored O: half an ulp of the largest magnitude in the row
     allowed = tol["o_max"] + ref["widen_o"]
+    if allow_output_rounding:
+        allowed = allowed + np.abs(ref["O"]).max(axis=-1) * 2.0 ** -8
     inf_both = np.isneginf(lse) & np.isneginf(ref["LSE"])
     err_l = np.where(inf_both, 0.0, np.abs(lse - ref["LSE"]))
     err_l = np.where(np.isnan(err_l), np.inf, err_l)

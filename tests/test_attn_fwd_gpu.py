@@ -50,6 +50,23 @@ def test_config1_gqa_peaked_rows(mode):
     assert st["ok"], st
 
 
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dtype", ["bf16", "fp8_e4m3"])
+def test_huge_score_range_reaches_the_clamp(mode, dtype):
+    # q and k scaled by 8 (exact in both storage types): offsets from the running maximum spread over
+    # hundreds of octaves, far below the h15 clamp at -126 and the pot floor at -20.
+    wl = Workload("wide", 1, 2, 1, 384, 384, 128, True, dtype, 43)
+    inp = make_inputs(wl)
+    if dtype == "bf16":
+        inp.q = (inp.q.float() * 8).to(torch.bfloat16)
+        inp.k = (inp.k.float() * 8).to(torch.bfloat16)
+    else:
+        inp.q_descale *= 8.0
+        inp.k_descale *= 8.0
+    st = compare(wl, mode, inp, allow_output_rounding=True)   # rows collapse onto single values of magnitude up to 4
+    assert st["ok"], st
+
+
 def test_fully_masked_rows_give_zero_and_minus_infinity():
     wl = Workload("masked", 1, 2, 2, 300, 100, 64, True, "bf16", 41)
     inp = make_inputs(wl)
