@@ -30,9 +30,8 @@ struct WsCfg {
     static constexpr int kQBytes = 2 * C::kTileBytes;
     static constexpr int kRingBytes = kSlots * C::kTileBytes;
     static constexpr int kScaleOff = kQBytes + kRingBytes;        // float alpha[2][128]
-    static constexpr int kFinalOff = kScaleOff + 2 * 128 * 4;     // float2 (l, m)[2][128]
-    static constexpr int kBarOff = kFinalOff + 2 * 128 * 8;
-    static constexpr int kNumBars = 2 + 2 * kSlots + 6 * 2 + 8;
+    static constexpr int kBarOff = kScaleOff + 2 * 128 * 4;
+    static constexpr int kNumBars = 2 * kSlots + 8 * 2;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kSmemBytes = kMiscOff + 16 + 1024;       // + manual 1024-byte alignment slack
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
@@ -54,13 +53,44 @@ __device__ __forceinline__ void reg_inc_192() { asm volatile("setmaxnreg.inc.syn
 #define ROWMAX_STAMP(role, j, slot) do { } while (0)
 #endif
 
-// Whether the two softmax warps of a scheduler alternate strictly (see the softmax role).  Measured
-// slower than free-running on every workload tried, so it is off; the barriers stay for experiments.
-constexpr bool kTakeTurns = false;
+// Tile 1 of a CTA's first work item starts once tile 0's first P is done, which spreads the two
+// tiles' softmax phases apart for the first iterations.
 constexpr bool kStagger = true;
 
-enum BarId : int { kBarQ = 0, kBarKvFull = 1, kBarKvEmpty = 2, kBarSFull = 3, kBarPFull = 4, kBarOFull = 5,
-                   kBarScale = 6, kBarORescaled = 7, kBarFinal = 8, kBarTurn = 9 };
+enum BarId : int { kBarQFull = 0, kBarQEmpty = 1, kBarKvFull = 2, kBarKvEmpty = 3, kBarSFull = 4, kBarPFull = 5,
+                   kBarOFull = 6, kBarScale = 7, kBarORescaled = 8, kBarOFree = 9 };
+
+// One work item = two query tiles of 128 rows of one (batch, head).
+struct WorkItem {
+    int h, b, hk;
+    int q0[2];   // first query row of each tile
+    int n[2];    // key tiles of each tile (0: the tile is out of range or sees no key)
+    int n_max;
+};
+
+// Items are numbered heaviest first (under a causal mask the last query tiles have the most key
+// tiles).  CTA c of G walks them in a snake: round k takes item k*G + c (k even) or k*G + G-1-c (k odd),
+// so every CTA gets one item of each weight class and the loads even out without a global counter.
+__device__ __forceinline__ int item_index(int round, int cta, int n_ctas) {
+    return round * n_ctas + ((round & 1) ? (n_ctas - 1 - cta) : cta);
+}
+__device__ __forceinline__ WorkItem decode_item(int w, const AttnParams& p, int n_pairs, int bh) {
+    WorkItem it;
+    const int pair = n_pairs - 1 - w / bh;
+    const int rem = w % bh;
+    it.h = rem % p.Hq;
+    it.b = rem / p.Hq;
+    it.hk = it.h / p.group;
+    const int shift = p.Sk - p.Sq;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        it.q0[t] = pair * 2 * kTileM + t * kTileM;
+        const int kv_end = p.causal ? min(p.Sk, it.q0[t] + kTileM + shift) : p.Sk;
+        it.n[t] = (it.q0[t] < p.Sq && kv_end > 0) ? (kv_end + kTileN - 1) / kTileN : 0;
+    }
+    it.n_max = max(it.n[0], it.n[1]);
+    return it;
+}
 
 }  // namespace
 
@@ -76,59 +106,47 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t sQ = smem_u32(smem);
     const uint32_t sRing = sQ + W::kQBytes;
     float* sScale = reinterpret_cast<float*>(smem + W::kScaleOff);
-    float2* sFinal = reinterpret_cast<float2*>(smem + W::kFinalOff);
     const uint32_t bar0 = smem_u32(smem + W::kBarOff);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + W::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + W::kMiscOff + 4);
     const WaitCtx wctx{abort_flag, p.status};
 
     // barrier addresses
-    auto bar_q = [&](int t) { return bar0 + 8u * t; };
-    auto bar_kv_full = [&](int s) { return bar0 + 8u * (2 + s); };
-    auto bar_kv_empty = [&](int s) { return bar0 + 8u * (2 + NS + s); };
-    auto bar_x = [&](int which, int t) { return bar0 + 8u * (2 + 2 * NS + 2 * which + t); };
-    auto bar_s_full = [&](int t) { return bar_x(0, t); };      // MMA -> softmax: S_t(j) is in TMEM
-    auto bar_p_full = [&](int t) { return bar_x(1, t); };      // softmax -> MMA: P_t(j) is in TMEM
-    auto bar_o_full = [&](int t) { return bar_x(2, t); };      // MMA -> correction: P_t V(j) accumulated
-    auto bar_scale = [&](int t) { return bar_x(3, t); };       // softmax -> correction: alpha_t(j) in smem
-    auto bar_o_rescaled = [&](int t) { return bar_x(4, t); };  // correction -> MMA: O_t rescaled for tile j
-    auto bar_final = [&](int t) { return bar_x(5, t); };       // softmax -> correction: (l, m) in smem
-    // turn token of the softmax warp pair that shares scheduler w: bar_turn(t, w) lets tile t's warp go
-    auto bar_turn = [&](int t, int w) { return bar0 + 8u * (2 + 2 * NS + 12 + 4 * t + w); };
+    auto bar_kv_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_kv_empty = [&](int s) { return bar0 + 8u * (NS + s); };
+    auto bar_x = [&](int which, int t) { return bar0 + 8u * (2 * NS + 2 * which + t); };
+    auto bar_q_full = [&](int t) { return bar_x(0, t); };      // TMA -> MMA: Q_t of the current item landed
+    auto bar_q_empty = [&](int t) { return bar_x(1, t); };     // MMA -> TMA: last S_t MMA of the item done
+    auto bar_s_full = [&](int t) { return bar_x(2, t); };      // MMA -> softmax: S_t(j) is in TMEM
+    auto bar_p_full = [&](int t) { return bar_x(3, t); };      // softmax -> MMA: P_t(j) is in TMEM
+    auto bar_o_full = [&](int t) { return bar_x(4, t); };      // MMA -> correction / epilogue: P_t V(j) accumulated
+    auto bar_scale = [&](int t) { return bar_x(5, t); };       // softmax -> correction: alpha_t(j) in smem
+    auto bar_o_rescaled = [&](int t) { return bar_x(6, t); };  // correction -> MMA: O_t rescaled for tile j
+    auto bar_o_free = [&](int t) { return bar_x(7, t); };      // epilogue -> MMA: O_t has been read out
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
+    if (tid == 256) ROWMAX_STAMP(2, 63, 0);
 
-    // work item: heaviest query tiles first (they have the most key tiles under a causal mask)
     const int n_pairs = (p.Sq + 2 * kTileM - 1) / (2 * kTileM);
     const int bh = p.Hq * p.B;
-    const int pair = n_pairs - 1 - static_cast<int>(blockIdx.x) / bh;
-    const int rem = static_cast<int>(blockIdx.x) % bh;
-    const int h = rem % p.Hq, b = rem / p.Hq, hk = h / p.group;
+    const int n_items = n_pairs * bh;
+    const int cta = blockIdx.x, n_ctas = gridDim.x;
     const int shift = p.Sk - p.Sq;
-    int q0t[2], n_t[2];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        q0t[t] = pair * 2 * kTileM + t * kTileM;
-        int kv_end = p.causal ? min(p.Sk, q0t[t] + kTileM + shift) : p.Sk;
-        n_t[t] = (q0t[t] < p.Sq && kv_end > 0) ? (kv_end + kTileN - 1) / kTileN : 0;
-    }
-    const int n_max = max(n_t[0], n_t[1]);
 
     if (tid == 0) {
-        mbar_init(bar_q(0), 1);
-        mbar_init(bar_q(1), 1);
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar_kv_full(s), 1);
             mbar_init(bar_kv_empty(s), 1);
         }
         for (int t = 0; t < 2; ++t) {
+            mbar_init(bar_q_full(t), 1);
+            mbar_init(bar_q_empty(t), 1);
             mbar_init(bar_s_full(t), 1);
             mbar_init(bar_p_full(t), 4);      // one arrival per softmax warp
             mbar_init(bar_o_full(t), 1);
             mbar_init(bar_scale(t), 4);
             mbar_init(bar_o_rescaled(t), 4);  // one arrival per correction warp
-            mbar_init(bar_final(t), 4);
-            for (int w = 0; w < 4; ++w) mbar_init(bar_turn(t, w), 1);
+            mbar_init(bar_o_free(t), 4);      // one arrival per softmax warp (epilogue)
         }
         *abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0);
         fence_mbar_init();
@@ -142,6 +160,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (tid == 256) ROWMAX_STAMP(2, 63, 1);
     auto tmem_S = [&](int t) { return tmem + 128u * t; };
     auto tmem_O = [&](int t) { return tmem + 256u + 128u * t; };
 
@@ -155,24 +174,39 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         reg_dec_48();
         if (warp == 13 && lane == 0) {
             // ------------------------------------------------------------ TMA producer
-            auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, uint32_t bar, int head, int row0) {
-                mbar_arrive_expect_tx(bar, C::kTileBytes);
+            int kv_idx = 0;             // K/V tiles loaded so far (ring position), over all items
+            int q_use[2] = {0, 0};      // items that used Q buffer t so far
+            for (int round = 0;; ++round) {
+                const int w = item_index(round, cta, n_ctas);
+                if (w >= n_items || *abort_flag) break;
+                const WorkItem it = decode_item(w, p, n_pairs, bh);
+                auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, uint32_t bar, int head, int row0) {
+                    mbar_arrive_expect_tx(bar, C::kTileBytes);
 #pragma unroll
-                for (int bx = 0; bx < C::kBoxes; ++bx)
-                    tma_load_4d(dst + bx * C::kBoxBytes, tm, bar, bx * C::kBoxElems, head, row0, b);
-            };
-            if (!*abort_flag) {
-                if (n_t[0] > 0) load_tile(&tmQ, sQ, bar_q(0), h, q0t[0]);
-                for (int j = 0; j < n_max; ++j) {
+                    for (int bx = 0; bx < C::kBoxes; ++bx)
+                        tma_load_4d(dst + bx * C::kBoxBytes, tm, bar, bx * C::kBoxElems, head, row0, it.b);
+                };
+                auto load_q = [&](int t) {
+                    if (it.n[t] > 0) {
+                        mbar_wait(bar_q_empty(t), (q_use[t] & 1) ^ 1, wctx, (kRoleLoad << 8) | kBarQEmpty);
+                        load_tile(&tmQ, sQ + t * C::kTileBytes, bar_q_full(t), it.h, it.q0[t]);
+                        ++q_use[t];
+                    }
+                };
+                if (round == 0) ROWMAX_STAMP(3, 63, 0);
+                load_q(0);
+                for (int j = 0; j < it.n_max; ++j) {
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
-                        const int idx = 2 * j + kv, slot = idx % NS, use = idx / NS;
+                        const int slot = kv_idx % NS, use = kv_idx / NS;
                         mbar_wait(bar_kv_empty(slot), (use & 1) ^ 1, wctx, (kRoleLoad << 8) | kBarKvEmpty);
-                        if (*abort_flag) break;
-                        load_tile(kv == 0 ? &tmK : &tmV, sRing + slot * C::kTileBytes, bar_kv_full(slot), hk, j * kTileN);
-                        if (j == 0 && kv == 0 && n_t[1] > 0) load_tile(&tmQ, sQ + C::kTileBytes, bar_q(1), h, q0t[1]);
+                        load_tile(kv == 0 ? &tmK : &tmV, sRing + slot * C::kTileBytes, bar_kv_full(slot), it.hk,
+                                  j * kTileN);
+                        ++kv_idx;
+                        if (j == 0 && kv == 0) load_q(1);
                     }
                 }
+                if (it.n_max == 0) load_q(1);
             }
         } else if (warp == 12) {
             // ------------------------------------------------------------ MMA issuer
@@ -204,273 +238,285 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             auto wait_full = [&](int idx) {
                 mbar_wait(bar_kv_full(idx % NS), (idx / NS) & 1, wctx, (kRoleMma << 8) | kBarKvFull);
             };
-            if (n_max > 0) {
-                wait_full(0);
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (n_t[t] > 0) {
-                        mbar_wait(bar_q(t), 0, wctx, (kRoleMma << 8) | kBarQ);
-                        // Stagger the two query tiles: tile 1 starts once tile 0's first P is done, which
-                        // spreads the two tiles' softmax phases apart for the first iterations.
-                        if (kStagger && t == 1 && n_t[0] > 0)
-                            mbar_wait(bar_p_full(0), 0, wctx, (kRoleMma << 8) | kBarPFull);
-                        tc_fence_after();
-                        if (leader) {
-                            if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(0));
-                            umma_commit(bar_s_full(t));
-                        }
-                    }
-                }
-                if (leader) umma_commit(bar_kv_empty(0));
-                for (int j = 0; j < n_max; ++j) {
-                    wait_full(2 * j + 1);
-                    bool k_ready = false;
+            int kv_base = 0;            // ring index of K_0 of the current item
+            int tiles[2] = {0, 0};      // key tiles of query tile t finished in earlier items (barrier phases)
+            int q_use[2] = {0, 0};      // items that used Q buffer / O accumulator t so far
+            for (int round = 0;; ++round) {
+                const int w = item_index(round, cta, n_ctas);
+                if (w >= n_items) break;
+                const WorkItem it = decode_item(w, p, n_pairs, bh);
+                if (it.n_max > 0) {
+                    wait_full(kv_base);
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
-                        if (j < n_t[t]) {
-                            mbar_wait(bar_p_full(t), j & 1, wctx, (kRoleMma << 8) | kBarPFull);
-                            if (leader) ROWMAX_STAMP(3, j, t * 4 + 0);
-                            mbar_wait(bar_o_rescaled(t), j & 1, wctx, (kRoleMma << 8) | kBarORescaled);
-                            if (leader) ROWMAX_STAMP(3, j, t * 4 + 1);
+                        if (it.n[t] > 0) {
+                            mbar_wait(bar_q_full(t), q_use[t] & 1, wctx, (kRoleMma << 8) | kBarQFull);
+                            if (kStagger && round == 0 && t == 1 && it.n[0] > 0)
+                                mbar_wait(bar_p_full(0), 0, wctx, (kRoleMma << 8) | kBarPFull);
                             tc_fence_after();
                             if (leader) {
-                                if (!*abort_flag) issue_pv(t, ring_lo_v + slot_lo(2 * j + 1), j > 0);
-                                umma_commit(bar_o_full(t));
-                                ROWMAX_STAMP(3, j, t * 4 + 2);
-                            }
-                        }
-                        if (j + 1 < n_t[t]) {
-                            if (!k_ready) {
-                                wait_full(2 * j + 2);
-                                tc_fence_after();
-                                k_ready = true;
-                            }
-                            if (leader) {
-                                if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(2 * j + 2));
+                                if (round == 0) ROWMAX_STAMP(3, 63, 1 + t);
+                                if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(kv_base));
                                 umma_commit(bar_s_full(t));
-                                ROWMAX_STAMP(3, j, t * 4 + 3);
+                                if (it.n[t] == 1) umma_commit(bar_q_empty(t));
                             }
                         }
                     }
-                    if (leader) {
-                        umma_commit(bar_kv_empty((2 * j + 1) % NS));
-                        if (j + 1 < n_max) umma_commit(bar_kv_empty((2 * j + 2) % NS));
+                    if (leader) umma_commit(bar_kv_empty(kv_base % NS));
+                    for (int j = 0; j < it.n_max; ++j) {
+                        wait_full(kv_base + 2 * j + 1);
+                        bool k_ready = false;
+#pragma unroll
+                        for (int t = 0; t < 2; ++t) {
+                            if (j < it.n[t]) {
+                                const uint32_t ph = (tiles[t] + j) & 1;
+                                mbar_wait(bar_p_full(t), ph, wctx, (kRoleMma << 8) | kBarPFull);
+                                if (leader) ROWMAX_STAMP(3, j, t * 4 + 0);
+                                mbar_wait(bar_o_rescaled(t), ph, wctx, (kRoleMma << 8) | kBarORescaled);
+                                // the accumulator of the previous item must have been read out
+                                if (j == 0) mbar_wait(bar_o_free(t), (q_use[t] & 1) ^ 1, wctx, (kRoleMma << 8) | kBarOFree);
+                                if (leader) ROWMAX_STAMP(3, j, t * 4 + 1);
+                                tc_fence_after();
+                                if (leader) {
+                                    if (!*abort_flag) issue_pv(t, ring_lo_v + slot_lo(kv_base + 2 * j + 1), j > 0);
+                                    umma_commit(bar_o_full(t));
+                                    ROWMAX_STAMP(3, j, t * 4 + 2);
+                                }
+                            }
+                            if (j + 1 < it.n[t]) {
+                                if (!k_ready) {
+                                    wait_full(kv_base + 2 * j + 2);
+                                    tc_fence_after();
+                                    k_ready = true;
+                                }
+                                if (leader) {
+                                    if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(kv_base + 2 * j + 2));
+                                    umma_commit(bar_s_full(t));
+                                    if (j + 2 == it.n[t]) umma_commit(bar_q_empty(t));   // last S of this item
+                                    ROWMAX_STAMP(3, j, t * 4 + 3);
+                                }
+                            }
+                        }
+                        if (leader) {
+                            umma_commit(bar_kv_empty((kv_base + 2 * j + 1) % NS));
+                            if (j + 1 < it.n_max) umma_commit(bar_kv_empty((kv_base + 2 * j + 2) % NS));
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
+                }
+                kv_base += 2 * it.n_max;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    tiles[t] += it.n[t];
+                    if (it.n[t] > 0) ++q_use[t];
                 }
             }
         }
     } else if (wg == 2) {
-        // ---------------------------------------------------------------- correction + epilogue
+        // ---------------------------------------------------------------- correction
         reg_dec_80();
         const int r = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        for (int j = 0; j < n_max; ++j) {
+        int tiles[2] = {0, 0};
+        for (int round = 0;; ++round) {
+            const int w = item_index(round, cta, n_ctas);
+            if (w >= n_items) break;
+            const WorkItem it = decode_item(w, p, n_pairs, bh);
+            for (int j = 0; j < it.n_max; ++j) {
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                if (j < n_t[t]) {
-                    mbar_wait(bar_scale(t), j & 1, wctx, (kRoleCorr << 8) | kBarScale);
-                    if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 0);
-                    const float alpha = sScale[t * 128 + r];
-                    if (j > 0) {
-                        mbar_wait(bar_o_full(t), (j - 1) & 1, wctx, (kRoleCorr << 8) | kBarOFull);
-                        if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 1);
-                        __syncwarp();
-                        tc_fence_after();
-                        if (__any_sync(0xffffffffu, alpha != 1.0f)) {
+                for (int t = 0; t < 2; ++t) {
+                    if (j < it.n[t]) {
+                        mbar_wait(bar_scale(t), (tiles[t] + j) & 1, wctx, (kRoleCorr << 8) | kBarScale);
+                        if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 0);
+                        const float alpha = sScale[t * 128 + r];
+                        if (j > 0) {
+                            mbar_wait(bar_o_full(t), (tiles[t] + j - 1) & 1, wctx, (kRoleCorr << 8) | kBarOFull);
+                            if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 1);
+                            __syncwarp();
+                            tc_fence_after();
+                            if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll
-                            for (int cc = 0; cc < D / 32; ++cc) {
-                                uint32_t o[32];
-                                tmem_ld32(tmem_O(t) + lane_base + cc * 32, o);
-                                tmem_wait_ld();
+                                for (int cc = 0; cc < D / 32; ++cc) {
+                                    uint32_t o[32];
+                                    tmem_ld32(tmem_O(t) + lane_base + cc * 32, o);
+                                    tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 32; i += 2) {
-                                    const float2 v = fmul2(make_float2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])),
-                                                           make_float2(alpha, alpha));
-                                    o[i] = __float_as_uint(v.x);
-                                    o[i + 1] = __float_as_uint(v.y);
+                                    for (int i = 0; i < 32; i += 2) {
+                                        const float2 v = fmul2(make_float2(__uint_as_float(o[i]), __uint_as_float(o[i + 1])),
+                                                               make_float2(alpha, alpha));
+                                        o[i] = __float_as_uint(v.x);
+                                        o[i + 1] = __float_as_uint(v.y);
+                                    }
+                                    tmem_st32(tmem_O(t) + lane_base + cc * 32, o);
                                 }
-                                tmem_st32(tmem_O(t) + lane_base + cc * 32, o);
+                                tmem_wait_st();
                             }
-                            tmem_wait_st();
+                            tc_fence_before();
                         }
-                        tc_fence_before();
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_o_rescaled(t));
-                    if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 2);
-                }
-            }
-        }
-        // epilogue: O = v_descale * acc / l (undoing the P offset), LSE = ln2 * (m c + log2 l)
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int row = q0t[t] + r;
-            if (q0t[t] >= p.Sq) continue;
-            float l_run = 0.f, m_run = -INFINITY;
-            if (n_t[t] > 0) {
-                mbar_wait(bar_final(t), 0, wctx, (kRoleEpi << 8) | kBarFinal);
-                const float2 lm = sFinal[t * 128 + r];
-                l_run = lm.x;
-                m_run = lm.y;
-                mbar_wait(bar_o_full(t), (n_t[t] - 1) & 1, wctx, (kRoleEpi << 8) | kBarOFull);
-                __syncwarp();
-                tc_fence_after();
-            }
-            const bool has_keys = l_run > 0.f;
-            const float inv = has_keys ? p.v_descale / l_run : 0.f;
-            if (row < p.Sq && p.lse != nullptr) {
-                const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - p_off) : -INFINITY;
-                p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.Sq + row] = lse;
-            }
-            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
-                                  ((static_cast<size_t>(b) * p.Sq + row) * p.Hq + h) * D;
-#pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) {
-                uint32_t o[32];
-                if (n_t[t] > 0) {
-                    tmem_ld32(tmem_O(t) + lane_base + cc * 32, o);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = 0;
-                }
-                if (row < p.Sq) {
-#pragma unroll
-                    for (int v4 = 0; v4 < 4; ++v4) {
-                        uint4 pk;
-                        pk.x = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
-                        pk.y = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
-                        pk.z = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
-                        pk.w = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + cc * 32 + v4 * 8) = pk;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_o_rescaled(t));
+                        if (r == 0) ROWMAX_STAMP(2, j, t * 4 + 2);
                     }
                 }
             }
+            tiles[0] += it.n[0];
+            tiles[1] += it.n[1];
         }
     } else {
-        // ---------------------------------------------------------------- softmax of query tile t
+        // ---------------------------------------------------------------- softmax + epilogue of query tile t
         reg_inc_192();
         const int t = wg;
         const int r = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_S(t) + lane_base;
-        const int q0 = t == 0 ? q0t[0] : q0t[1];
-        const int nt = t == 0 ? n_t[0] : n_t[1];
-        // The two softmax warps on one scheduler take turns on their arithmetic-heavy section, tile by
-        // tile (0, 1, 0, 1, ...), so that each runs it alone and the two query tiles stay half a period
-        // apart: while one warp computes weights, the other's MMAs and hand-offs are in flight.
-        const int n_both = kTakeTurns ? min(n_t[0], n_t[1]) : 0;   // tiles for which both warps are active
-        const int w4 = warp & 3;
-        const int row = q0 + r;
-        const int row_limit = p.causal ? min(p.Sk, row + shift + 1) : p.Sk;  // visible keys of this row
-        // first key index that some row of this tile cannot see (tile-uniform)
-        const int tile_limit = p.causal ? min(p.Sk, q0 + shift + 1) : p.Sk;
+        const uint32_t tO = tmem_O(t) + lane_base;
         const float c_eff = (MODE == kH15) ? 2.0f * p.c : p.c;
-        float m_run = -INFINITY, l_run = 0.f;
-        for (int j = 0; j < nt; ++j) {
-            mbar_wait(bar_s_full(t), j & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);
-            if (t == 0) {
-                if (j > 0 && j < n_both) mbar_wait(bar_turn(0, w4), (j - 1) & 1, wctx, (kRoleSoftmax << 8) | kBarTurn);
-            } else {
-                if (j < n_both) mbar_wait(bar_turn(1, w4), j & 1, wctx, (kRoleSoftmax << 8) | kBarTurn);
-            }
-            if (r == 0) ROWMAX_STAMP(t, j, 0);
-            __syncwarp();
-            tc_fence_after();
-            uint32_t s[4][32];
+        int tiles = 0;
+        for (int round = 0;; ++round) {
+            const int w = item_index(round, cta, n_ctas);
+            if (w >= n_items) break;
+            const WorkItem it = decode_item(w, p, n_pairs, bh);
+            const int q0 = t == 0 ? it.q0[0] : it.q0[1];
+            const int nt = t == 0 ? it.n[0] : it.n[1];
+            const int row = q0 + r;
+            const int row_limit = p.causal ? min(p.Sk, row + shift + 1) : p.Sk;  // visible keys of this row
+            // first key index that some row of this tile cannot see (tile-uniform)
+            const int tile_limit = p.causal ? min(p.Sk, q0 + shift + 1) : p.Sk;
+            float m_run = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < nt; ++j) {
+                mbar_wait(bar_s_full(t), (tiles + j) & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);
+                if (r == 0) ROWMAX_STAMP(t, j, 0);
+                __syncwarp();
+                tc_fence_after();
+                uint32_t s[4][32];
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, s[cc]);
-            tmem_wait_ld();
-            if (r == 0) ROWMAX_STAMP(t, j, 1);
+                for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, s[cc]);
+                tmem_wait_ld();
+                if (r == 0) ROWMAX_STAMP(t, j, 1);
 
-            const bool masked_tile = (j + 1) * kTileN > tile_limit;
-            const int col_limit = row_limit - j * kTileN;
-            if (masked_tile) {
+                const bool masked_tile = (j + 1) * kTileN > tile_limit;
+                const int col_limit = row_limit - j * kTileN;
+                if (masked_tile) {
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
+                    for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (cc * 32 + i >= col_limit) s[cc][i] = __float_as_uint(-INFINITY);
-            }
-            const float m_t = row_max128(s);
-            const float m_new = fmaxf(m_run, m_t);
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-            const float alpha = ex2_approx((m_run - m_use) * p.c);
-            m_run = m_new;
-            sScale[t * 128 + r] = alpha;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_scale(t));
-            if (r == 0) ROWMAX_STAMP(t, j, 2);
+                        for (int i = 0; i < 32; ++i)
+                            if (cc * 32 + i >= col_limit) s[cc][i] = __float_as_uint(-INFINITY);
+                }
+                const float m_t = row_max128(s);
+                const float m_new = fmaxf(m_run, m_t);
+                const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+                const float alpha = ex2_approx((m_run - m_use) * p.c);
+                m_run = m_new;
+                sScale[t * 128 + r] = alpha;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_scale(t));
+                if (r == 0) ROWMAX_STAMP(t, j, 2);
 
-            // exact: x = s*c - m*c + P offset;  h15: doubled input 2x = s*(2c) - m*(2c);  pot: x = s*c - m*c
-            RowScale rs;
-            rs.c = make_float2(c_eff, c_eff);
-            const float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
-            rs.nmc = make_float2(nmc, nmc);
-            rs.two22 = p.two22;
-            float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-            if (masked_tile) {
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t pw[16];
-                    weights_chunk32<FP8, MODE, true>(s[cc], rs, col_limit - cc * 32, acc, pw);
-                    if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
-                    else tmem_st16(tS + cc * 16, pw);
-                }
-            } else {
-                // h15: the clamp at -252 is a no-op unless some score of the warp's rows lies more than
-                // 126 octaves below its running maximum; the row minimum (one more three-input pass)
-                // tells, and the common case runs without the per-score clamp.
-                bool clamp = false;
-                if constexpr (MODE == kH15) {
-                    const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest doubled offset of the row
-                    clamp = __any_sync(0xffffffffu, !(lowest >= -250.0f));
-                }
-                if (clamp) {
+                // exact: x = s*c - m*c + P offset;  h15: doubled input 2x = s*(2c) - m*(2c);  pot: x = s*c - m*c
+                RowScale rs;
+                rs.c = make_float2(c_eff, c_eff);
+                const float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
+                rs.nmc = make_float2(nmc, nmc);
+                rs.two22 = p.two22;
+                float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                if (masked_tile) {
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t pw[16];
-                        weights_chunk32<FP8, MODE, false, true>(s[cc], rs, 32, acc, pw);
+                        weights_chunk32<FP8, MODE, true>(s[cc], rs, col_limit - cc * 32, acc, pw);
                         if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                         else tmem_st16(tS + cc * 16, pw);
                     }
                 } else {
+                    // h15: the clamp at -252 is a no-op unless some score of the warp's rows lies more than
+                    // 126 octaves below its running maximum; the row minimum (one more three-input pass)
+                    // tells, and the common case runs without the per-score clamp.
+                    bool clamp = false;
+                    if constexpr (MODE == kH15) {
+                        const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest doubled offset of the row
+                        clamp = __any_sync(0xffffffffu, !(lowest >= -250.0f));
+                    }
+                    if (clamp) {
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t pw[16];
-                        weights_chunk32<FP8, MODE, false, false>(s[cc], rs, 32, acc, pw);
-                        if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
-                        else tmem_st16(tS + cc * 16, pw);
+                        for (int cc = 0; cc < 4; ++cc) {
+                            uint32_t pw[16];
+                            weights_chunk32<FP8, MODE, false, true>(s[cc], rs, 32, acc, pw);
+                            if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
+                            else tmem_st16(tS + cc * 16, pw);
+                        }
+                    } else {
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) {
+                            uint32_t pw[16];
+                            weights_chunk32<FP8, MODE, false, false>(s[cc], rs, 32, acc, pw);
+                            if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
+                            else tmem_st16(tS + cc * 16, pw);
+                        }
+                    }
+                }
+                const float l_tile = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
+                if (r == 0) ROWMAX_STAMP(t, j, 3);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p_full(t));
+                if (r == 0) ROWMAX_STAMP(t, j, 4);
+                l_run = l_run * alpha + l_tile;
+            }
+
+            // epilogue of this tile: O = v_descale * acc / l (the P offset cancels), LSE = ln2 * (m c + log2 l)
+            if (q0 < p.Sq) {
+                const bool has_keys = l_run > 0.f;
+                const float inv = has_keys ? p.v_descale / l_run : 0.f;
+                if (row < p.Sq && p.lse != nullptr) {
+                    const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - p_off) : -INFINITY;
+                    p.lse[(static_cast<size_t>(it.b) * p.Hq + it.h) * p.Sq + row] = lse;
+                }
+                if (nt > 0) {
+                    mbar_wait(bar_o_full(t), (tiles + nt - 1) & 1, wctx, (kRoleEpi << 8) | kBarOFull);
+                    __syncwarp();
+                    tc_fence_after();
+                }
+                if (r == 0 && round == 0) ROWMAX_STAMP(2, 63, 2 + 2 * t);
+                __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
+                                      ((static_cast<size_t>(it.b) * p.Sq + row) * p.Hq + it.h) * D;
+#pragma unroll
+                for (int cc = 0; cc < D / 32; ++cc) {
+                    uint32_t o[32];
+                    if (nt > 0) {
+                        tmem_ld32(tO + cc * 32, o);
+                        tmem_wait_ld();
+                        if (cc == D / 32 - 1) {   // the accumulator is in registers: the next item may overwrite it
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_o_free(t));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = 0;
+                    }
+                    if (row < p.Sq) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint4 pk;
+                            pk.x = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
+                            pk.y = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
+                            pk.z = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
+                            pk.w = pack_bf16_rn(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
+                            *reinterpret_cast<uint4*>(orow + cc * 32 + v4 * 8) = pk;
+                        }
                     }
                 }
             }
-            const float l_tile = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
-            if (r == 0) ROWMAX_STAMP(t, j, 3);
-            __syncwarp();
-            if (lane == 0) {   // pass the turn to the other tile's warp
-                if (t == 0) {
-                    if (j < n_both) mbar_arrive(bar_turn(1, w4));
-                } else {
-                    if (j + 1 < n_both) mbar_arrive(bar_turn(0, w4));
-                }
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_p_full(t));
-            if (r == 0) ROWMAX_STAMP(t, j, 4);
-            l_run = l_run * alpha + l_tile;
-        }
-        if (nt > 0) {
-            sFinal[t * 128 + r] = make_float2(l_run, m_run);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_final(t));
+            tiles += nt;
         }
     }
 
+    if (tid == 256) ROWMAX_STAMP(2, 63, 6);
     tc_fence_before();
     __syncthreads();
+    if (tid == 256) ROWMAX_STAMP(2, 63, 7);
     if (warp == 12) tmem_dealloc(tmem, kTmemCols);
 }
 
@@ -489,9 +535,18 @@ static cudaError_t launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const
         configured = true;
     }
     const long long n_pairs = (p.Sq + 2 * kTileM - 1) / (2 * kTileM);
-    const long long blocks = n_pairs * p.Hq * p.B;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<static_cast<unsigned>(blocks), 512, W::kSmemBytes, stream>>>(tq, tk, tv, p);
+    const long long items = n_pairs * p.Hq * p.B;
+    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
+    // persistent CTAs: one per SM (shared memory and TMEM allow no more), each walking its share of the items
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+    }
+    const unsigned blocks = static_cast<unsigned>(items < sm_count ? items : sm_count);
+    kern<<<blocks, 512, W::kSmemBytes, stream>>>(tq, tk, tv, p);
     return cudaGetLastError();
 }
 
