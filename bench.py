@@ -35,7 +35,7 @@ TWIN = WORKLOADS[3]           # non-causal 8K fp8
 METRIC = "attn_fwd_tflops_h15_causal_8k_fp8"
 # dram__bytes_read.sum + dram__bytes_write.sum of one h15 launch on the headline workload, from the ncu
 # capture summarised in profiles/attn_fwd_ws_causal_8k_fp8.txt (algorithmic: 101 MB in + 68 MB out)
-NCU_DRAM_BYTES_PER_LAUNCH = 169.6e6 + 32.4e6
+NCU_DRAM_BYTES_PER_LAUNCH = 170.2e6 + 33.2e6
 MODE_IDS = {"exact": 0, "pot": 1, "h15": 2}
 
 
@@ -169,7 +169,7 @@ def oracle_sample(wl: Workload, inp, mode: int, row_stride: int, n_batch=None, n
             "pairs": sub.B * sub.Hq}
 
 
-def cpu_baseline_leg(wl: Workload, inp, row_stride: int = 8):
+def cpu_baseline_leg(wl: Workload, inp, row_stride: int = 4):
     s = oracle_sample(wl, inp, MODE_IDS["h15"], row_stride)
     return {"value": s["flops"] / s["seconds"] / 1e12, "unit": "TFLOP/s", "cores": s["threads"], "kind": "oracle",
             "sample": f"every {row_stride}th query row of {wl.name} ({s['rows']} rows x {s['pairs']} (batch, head) "
