@@ -45,8 +45,29 @@ def test_small_shapes(wl, mode):
 @pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_H15])
 def test_config1_gqa_peaked_rows(mode):
     wl = WORKLOADS[1]
-    rows = np.unique(np.concatenate([np.arange(0, wl.Sq, 16), np.arange(128), np.arange(wl.Sq - 128, wl.Sq)]))
-    st = compare(wl, mode, rows=rows)
+    st = compare(wl, mode, rows=_sample_rows(wl.Sq, 16))
+    assert st["ok"], st
+
+
+def _sample_rows(S, stride):
+    """Every stride-th row, plus all rows of the first and the last query tile."""
+    return np.unique(np.concatenate([np.arange(0, S, stride), np.arange(128), np.arange(S - 128, S)]))
+
+
+@pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_H15])
+@pytest.mark.parametrize("idx", [2, 3])
+def test_config2_and_3_full_size_8k_fp8_on_sampled_rows(idx, mode):
+    # the workloads and launch configuration bench.py times; the oracle computes sampled rows one by one
+    wl = WORKLOADS[idx]
+    st = compare(wl, mode, rows=_sample_rows(wl.Sq, 128))
+    assert st["ok"], st
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dtype", ["bf16", "fp8_e4m3"])
+def test_config4_full_size_16k_gqa_on_sampled_rows(dtype, mode):
+    wl = WORKLOADS[4].with_(in_dtype=dtype)
+    st = compare(wl, mode, rows=_sample_rows(wl.Sq, 512))
     assert st["ok"], st
 
 
