@@ -264,36 +264,31 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     }
                     if (leader) umma_commit(bar_kv_empty(kv_base % NS));
                     for (int j = 0; j < it.n_max; ++j) {
+                        // Everything the next MMAs need besides P is awaited first (it is normally there long
+                        // before), so that once P_t(j) arrives the P V and next-S MMAs go out back to back.
+                        const bool ok = !*abort_flag;
                         wait_full(kv_base + 2 * j + 1);
-                        bool k_ready = false;
+                        if (j + 1 < it.n_max) wait_full(kv_base + 2 * j + 2);
 #pragma unroll
                         for (int t = 0; t < 2; ++t) {
                             if (j < it.n[t]) {
                                 const uint32_t ph = (tiles[t] + j) & 1;
-                                mbar_wait(bar_p_full(t), ph, wctx, (kRoleMma << 8) | kBarPFull);
-                                if (leader) ROWMAX_STAMP(3, j, t * 4 + 0);
                                 mbar_wait(bar_o_rescaled(t), ph, wctx, (kRoleMma << 8) | kBarORescaled);
                                 // the accumulator of the previous item must have been read out
                                 if (j == 0) mbar_wait(bar_o_free(t), (q_use[t] & 1) ^ 1, wctx, (kRoleMma << 8) | kBarOFree);
-                                if (leader) ROWMAX_STAMP(3, j, t * 4 + 1);
+                                mbar_wait(bar_p_full(t), ph, wctx, (kRoleMma << 8) | kBarPFull);
+                                if (leader) ROWMAX_STAMP(3, j, t * 4 + 0);
                                 tc_fence_after();
                                 if (leader) {
-                                    if (!*abort_flag) issue_pv(t, ring_lo_v + slot_lo(kv_base + 2 * j + 1), j > 0);
+                                    if (ok) issue_pv(t, ring_lo_v + slot_lo(kv_base + 2 * j + 1), j > 0);
                                     umma_commit(bar_o_full(t));
                                     ROWMAX_STAMP(3, j, t * 4 + 2);
-                                }
-                            }
-                            if (j + 1 < it.n[t]) {
-                                if (!k_ready) {
-                                    wait_full(kv_base + 2 * j + 2);
-                                    tc_fence_after();
-                                    k_ready = true;
-                                }
-                                if (leader) {
-                                    if (!*abort_flag) issue_s(t, ring_lo_k + slot_lo(kv_base + 2 * j + 2));
-                                    umma_commit(bar_s_full(t));
-                                    if (j + 2 == it.n[t]) umma_commit(bar_q_empty(t));   // last S of this item
-                                    ROWMAX_STAMP(3, j, t * 4 + 3);
+                                    if (j + 1 < it.n[t]) {
+                                        if (ok) issue_s(t, ring_lo_k + slot_lo(kv_base + 2 * j + 2));
+                                        umma_commit(bar_s_full(t));
+                                        if (j + 2 == it.n[t]) umma_commit(bar_q_empty(t));   // last S of this item
+                                        ROWMAX_STAMP(3, j, t * 4 + 3);
+                                    }
                                 }
                             }
                         }
