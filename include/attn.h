@@ -72,6 +72,21 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
              float q_descale, float k_descale, float v_descale, void* stream);
 
 /*
+ * attn_fwd_tau — attn_fwd with a deferred rescale (App. B "Conditional rescaling moves the anchor";
+ * the rule of the paper's BF16 kernel, which uses rescale_tau = 8): a key tile's maximum replaces the
+ * row's anchor only when it exceeds the anchor by more than rescale_tau octaves of the scaled score,
+ * so O is rescaled far less often and x can be positive (Eq. h15 covers both signs).  Exact mode is
+ * unchanged by this up to rounding; pot and h15 results differ from rescale_tau = 0 because the
+ * lattice is anchored at the lagging maximum.  bf16 inputs only (ATTN_ERR_UNSUPPORTED for fp8: its P
+ * formats have no headroom above the anchor); 0 <= rescale_tau <= 32, else ATTN_ERR_BAD_VALUE.
+ * attn_fwd is attn_fwd_tau with rescale_tau = 0.
+ */
+int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* lse,
+                 int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                 int causal, float softmax_scale, int weight_mode, int in_dtype,
+                 float q_descale, float k_descale, float v_descale, float rescale_tau, void* stream);
+
+/*
  * attn_weight_map — applies the weight map of `weight_mode` to n fp32 offsets with the same device
  * function the fused kernel uses (Eq. m-exact / Eq. rowmax-pot / Eq. h15; the h15 input is clamped
  * below at -126, App. B.1 "Implementation").  x and w are device arrays of n floats; they may alias.
@@ -86,7 +101,8 @@ int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* s
  * Host-only query, no CUDA call.  Any output pointer may be NULL.
  *   tile_m, tile_n   query rows / keys per tile
  *   kv_order         +1: key tiles visited in ascending order
- *   rescale_tau      running-maximum adoption threshold in octaves (0 = the anchor is always current)
+ *   rescale_tau      anchor adoption threshold in octaves used by attn_fwd (0 = the anchor is always current);
+ *                    attn_fwd_tau takes its own
  *   pot_kmax         K_max of Rowmax-PoT
  *   p_format         ATTN_P_*; p_offset_log2: P is stored as weight * 2^p_offset_log2
  */

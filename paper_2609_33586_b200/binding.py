@@ -19,7 +19,7 @@ MODES = {"exact": W_EXACT, "pot": W_POT, "h15": W_H15}
 _LIB_PATH = Path(__file__).resolve().parent / "libattn_b200.so"
 _lib = None
 
-EXPORTS = ("attn_fwd", "attn_weight_map", "attn_get_schedule", "attn_device_status",
+EXPORTS = ("attn_fwd", "attn_fwd_tau", "attn_weight_map", "attn_get_schedule", "attn_device_status",
            "attn_device_status_reset", "attn_launch_count", "attn_status_string",
            "attn_last_cuda_error", "attn_version")
 
@@ -41,6 +41,8 @@ def lib() -> ctypes.CDLL:
         vp, i, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
         L.attn_fwd.restype = i
         L.attn_fwd.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, f, f, f, vp]
+        L.attn_fwd_tau.restype = i
+        L.attn_fwd_tau.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, f, f, f, f, vp]
         L.attn_weight_map.restype = i
         L.attn_weight_map.argtypes = [vp, vp, ctypes.c_size_t, i, vp]
         L.attn_get_schedule.restype = i
@@ -106,19 +108,25 @@ def in_dtype_of(t: torch.Tensor) -> int:
 
 
 def attn_fwd_raw(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale,
-                 weight_mode, in_dtype, q_descale, k_descale, v_descale, stream_ptr) -> int:
-    """Direct call with integer device addresses; returns the status code."""
-    return lib().attn_fwd(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
-                          softmax_scale, weight_mode, in_dtype, q_descale, k_descale, v_descale,
-                          stream_ptr)
+                 weight_mode, in_dtype, q_descale, k_descale, v_descale, stream_ptr, rescale_tau=None) -> int:
+    """Direct call with integer device addresses; returns the status code.  With `rescale_tau` the
+    call goes to attn_fwd_tau."""
+    if rescale_tau is None:
+        return lib().attn_fwd(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
+                              softmax_scale, weight_mode, in_dtype, q_descale, k_descale, v_descale,
+                              stream_ptr)
+    return lib().attn_fwd_tau(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
+                              softmax_scale, weight_mode, in_dtype, q_descale, k_descale, v_descale,
+                              rescale_tau, stream_ptr)
 
 
 def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool, softmax_scale: float,
              weight_mode: int, q_descale: float = 1.0, k_descale: float = 1.0, v_descale: float = 1.0,
              out: torch.Tensor | None = None, lse: torch.Tensor | None = None, return_lse: bool = True,
-             stream=None):
+             rescale_tau: float | None = None, stream=None):
     """q (B,Sq,Hq,D), k/v (B,Sk,Hkv,D): contiguous CUDA tensors, bf16 or float8_e4m3fn.
-    Returns (O bf16 (B,Sq,Hq,D), LSE fp32 (B,Hq,Sq) or None)."""
+    Returns (O bf16 (B,Sq,Hq,D), LSE fp32 (B,Hq,Sq) or None).  `rescale_tau` (bf16 inputs only) selects
+    the deferred-rescale entry point attn_fwd_tau."""
     for t in (q, k, v):
         if not t.is_cuda or not t.is_contiguous():
             raise ValueError("q, k, v must be contiguous CUDA tensors")
@@ -136,7 +144,7 @@ def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool,
     rc = attn_fwd_raw(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                       lse.data_ptr() if lse is not None else None, B, Hq, Hkv, Sq, Sk, D, causal,
                       softmax_scale, weight_mode, dt, q_descale, k_descale, v_descale,
-                      _stream_ptr(stream))
+                      _stream_ptr(stream), rescale_tau)
     if rc != 0:
         raise AttnError(rc, "attn_fwd")
     return out, lse

@@ -112,9 +112,9 @@ void attn_set_trace(long long* device_buffer, int block) {
 }
 #endif
 
-int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
-             int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
-             float k_descale, float v_descale, void* stream) {
+int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+                 int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
+                 float k_descale, float v_descale, float rescale_tau, void* stream) {
     if (!q || !k || !v || !o) return ATTN_ERR_NULLPTR;
     if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15) return ATTN_ERR_BAD_ENUM;
     if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
@@ -129,6 +129,8 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
         return ATTN_ERR_BAD_VALUE;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return ATTN_ERR_MISALIGNED;
     if (fp8 && D != 128) return ATTN_ERR_UNSUPPORTED;
+    if (!(rescale_tau >= 0.f) || !std::isfinite(rescale_tau) || rescale_tau > 32.f) return ATTN_ERR_BAD_VALUE;
+    if (fp8 && rescale_tau != 0.f) return ATTN_ERR_UNSUPPORTED;   // the fp8 P formats have no headroom above the anchor
     int rc = check_arch();
     if (rc != ATTN_OK) return rc;
 
@@ -143,6 +145,7 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
     p.c = static_cast<float>(static_cast<double>(softmax_scale) * dq * dk * 1.4426950408889634074);
     p.v_descale = fp8 ? v_descale : 1.0f;
     p.two22 = 1u << 22;
+    p.tau = rescale_tau;
 #ifdef ROWMAX_TRACE
     p.trace = g_trace;
     p.trace_block = g_trace_block;
@@ -162,6 +165,13 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return ATTN_OK;
+}
+
+int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+             int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
+             float k_descale, float v_descale, void* stream) {
+    return attn_fwd_tau(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale, weight_mode, in_dtype,
+                        q_descale, k_descale, v_descale, 0.0f, stream);
 }
 
 int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* stream) {

@@ -399,7 +399,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                             if (cc * 32 + i >= col_limit) s[cc][i] = __float_as_uint(-INFINITY);
                 }
                 const float m_t = row_max128(s);
-                const float m_new = fmaxf(m_run, m_t);
+                // The tile maximum becomes the new anchor when there is none yet or when it exceeds the
+                // anchor by more than tau octaves (tau = 0: always, so the anchor is the running maximum).
+                const bool adopt = (m_run == -INFINITY) || ((m_t - m_run) * p.c > p.tau);
+                const float m_new = adopt ? fmaxf(m_run, m_t) : m_run;
                 const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
                 const float alpha = ex2_approx((m_run - m_use) * p.c);
                 m_run = m_new;

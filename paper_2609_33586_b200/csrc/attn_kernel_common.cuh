@@ -18,6 +18,7 @@ struct AttnParams {
     int group;        // Hq / Hkv
     float c;          // softmax_scale * q_descale * k_descale * log2(e), rounded once to fp32
     float v_descale;  // 1 for bf16
+    float tau;        // rescale threshold in octaves (0 = the anchor is always the running maximum)
     uint32_t two22;   // 1 << 22, kept in a register for the h15 integer multiply-add
     int* status;      // device-global sticky status word
 #ifdef ROWMAX_TRACE

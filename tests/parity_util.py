@@ -27,18 +27,21 @@ EXACT_FP8_FEW_KEYS = 16
 EXACT_FP8_FEW_KEYS_TOL = 1e-1
 
 
-def run_cuda(wl: Workload, inp: Inputs, mode: int, device="cuda:0"):
+def run_cuda(wl: Workload, inp: Inputs, mode: int, device="cuda:0", tau=None):
     q, k, v = (t.to(device) for t in (inp.q, inp.k, inp.v))
     o, lse = binding.attn_fwd(q, k, v, causal=wl.causal, softmax_scale=wl.softmax_scale, weight_mode=mode,
-                              q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale)
+                              q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale,
+                              rescale_tau=tau)
     torch.cuda.synchronize()
     return o, lse
 
 
-def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None):
+def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None):
     dt = orc.IN_BF16 if wl.in_dtype == "bf16" else orc.IN_FP8_E4M3
     sch = binding.get_schedule(wl.D, dt, mode, wl.causal)
     assert sch["rescale_tau"] == 0.0
+    if tau is not None:
+        sch["rescale_tau"] = tau
     tile = 0 if mode == orc.W_EXACT else sch["tile_n"]   # exact mode: the whole-row definition
     return orc.attn(storage_bits(inp.q), storage_bits(inp.k), storage_bits(inp.v), in_dtype=dt,
                     causal=wl.causal, softmax_scale=wl.softmax_scale, mode=mode, tile_n=tile,
@@ -48,15 +51,15 @@ def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None):
 
 
 def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, device="cuda:0",
-            allow_output_rounding: bool = False):
+            allow_output_rounding: bool = False, tau=None):
     """Returns a dict of error statistics; `ok` says whether every gate holds.
 
     `allow_output_rounding` adds half a bf16 ulp of the reference value to the per-row tolerance: O
     is stored in bf16, and for outputs of magnitude 2 and above that rounding alone is 0.008 and
     more.  The standard workloads (N(0,1) values, averaged) do not need it."""
     inp = inp or make_inputs(wl)
-    o, lse = run_cuda(wl, inp, mode, device)
-    ref = run_oracle(wl, inp, mode, rows)
+    o, lse = run_cuda(wl, inp, mode, device, tau)
+    ref = run_oracle(wl, inp, mode, rows, tau)
     o = o.float().cpu().numpy().transpose(0, 2, 1, 3).astype(np.float64)   # (B,Hq,Sq,D)
     lse = lse.cpu().numpy().astype(np.float64)
     if rows is not None:

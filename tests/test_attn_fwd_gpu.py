@@ -88,6 +88,28 @@ def test_huge_score_range_reaches_the_clamp(mode, dtype):
     assert st["ok"], st
 
 
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("tau", [8.0, 2.0])
+def test_deferred_rescale_matches_the_oracle_with_the_same_threshold(mode, tau):
+    # the anchor lags the running maximum by up to tau octaves: x can be positive, weights exceed 1
+    # (in exact mode the largest weight of a row is then 2^x with x > 0 instead of exactly 1, so its bf16
+    # rounding, 2^-9 relative, shows in peaked rows: allow it on top of the bf16 rounding of O itself)
+    wl = Workload("tau", 2, 4, 2, 600, 600, 128, True, "bf16", 44, peaked_keys=True)
+    st = compare(wl, mode, tau=tau, allow_output_rounding=True)
+    assert st["ok"], st
+    wl64 = Workload("tau64", 1, 2, 2, 384, 512, 64, False, "bf16", 45)
+    st = compare(wl64, mode, tau=tau, allow_output_rounding=True)
+    assert st["ok"], st
+
+
+def test_deferred_rescale_is_rejected_for_fp8_and_bad_values():
+    q = torch.zeros(1, 128, 2, 128, dtype=torch.bfloat16, device="cuda")
+    args = (q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128, 128, 1, 0.1, 2)
+    assert binding.attn_fwd_raw(*args, 1, 1.0, 1.0, 1.0, None, rescale_tau=8.0) == -8     # fp8
+    assert binding.attn_fwd_raw(*args, 0, 1.0, 1.0, 1.0, None, rescale_tau=-1.0) == -9
+    assert binding.attn_fwd_raw(*args, 0, 1.0, 1.0, 1.0, None, rescale_tau=float("nan")) == -9
+
+
 def test_fully_masked_rows_give_zero_and_minus_infinity():
     wl = Workload("masked", 1, 2, 2, 300, 100, 64, True, "bf16", 41)
     inp = make_inputs(wl)
