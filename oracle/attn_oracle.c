@@ -13,6 +13,8 @@
  *   - Rowmax-H15: n = RNE(2x), w = (1 + (n mod 2)/2) * 2^floor(n/2) .......... Eq. m-h15 (Sec. 5.2), Eq. h15 (App. B.1)
  *   - lower clamp of the H15 input at x = -126 (doubled input at -252) ...... App. B.1 "Implementation",
  *                                                                            App. B "Exponential-map ablation"
+ *   - the H15 family S(Q_{2^-k}(x)), k = 2, 3 ................................. App. B "Exponential-map ablation",
+ *                                                                            App. B.1 "Relation to classical bit-level exponentiation"
  *   - anchor = the running row maximum of the online loop, tile of 128 keys,
  *     rescale rule, per-row decision; row sum and PV use the same weights ... Sec. 5.2, App. B.1,
  *                                                                            App. B "Semantic simulation"
@@ -34,7 +36,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_W_EXACT = 0, ORACLE_W_POT = 1, ORACLE_W_H15 = 2 };
+enum { ORACLE_W_EXACT = 0, ORACLE_W_POT = 1, ORACLE_W_H15 = 2, ORACLE_W_H15K2 = 3, ORACLE_W_H15K3 = 4 };
 enum { ORACLE_IN_BF16 = 0, ORACLE_IN_FP8_E4M3 = 1 };
 enum { ORACLE_P_NONE = 0, ORACLE_P_BF16 = 1, ORACLE_P_E4M3 = 2, ORACLE_P_E5M2 = 3 };
 
@@ -131,17 +133,33 @@ double oracle_w_h15(float x) {
     return (1.0 + 0.5 * b) * ldexp(1.0, (int)k);
 }
 
+/* The family Rowmax-H15 belongs to (App. B "Exponential-map ablation"): the unshifted Schraudolph
+ * construction S(q) = 2^floor(q) (1 + q - floor(q)) evaluated on the input rounded to steps of 2^-k,
+ * q = RNE(2^k x) / 2^k, after the same lower clamp max(x, -126).  k = 1 is Rowmax-H15 itself;
+ * k = 2, 3 are the quarter- and eighth-octave members. */
+double oracle_w_h15_family(float x, int k) {
+    if (isnan(x)) return NAN;
+    double xd = (double)x;
+    if (xd < -126.0) xd = -126.0;
+    double steps = ldexp(1.0, k);
+    double q = nearbyint(steps * xd) / steps;
+    double fl = floor(q);
+    return ldexp(1.0 + (q - fl), (int)fl);
+}
+
 static double weight_of(float x, int mode, int kmax) {
     switch (mode) {
         case ORACLE_W_POT: return oracle_w_pot(x, kmax);
         case ORACLE_W_H15: return oracle_w_h15(x);
+        case ORACLE_W_H15K2: return oracle_w_h15_family(x, 2);
+        case ORACLE_W_H15K3: return oracle_w_h15_family(x, 3);
         default: return oracle_w_exact(x);
     }
 }
 
 /* Array form used by the sweep tests.  Returns 0, or -1 for a bad mode. */
 int oracle_weight_map(const float* x, double* w, size_t n, int mode, int kmax) {
-    if (mode < 0 || mode > 2) return -1;
+    if (mode < 0 || mode > 4) return -1;
     fesetround(FE_TONEAREST);
     for (size_t i = 0; i < n; ++i) w[i] = weight_of(x[i], mode, kmax);
     return 0;
@@ -266,8 +284,9 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
             for (int d = 0; d < D; ++d) o[d] += pw * vr[d];
             if (mode != ORACLE_W_EXACT && tie_eps > 0.0) {
                 double u, dist;
-                if (mode == ORACLE_W_H15) {
-                    u = 2.0 * ((double)x < -126.0 ? -126.0 : (double)x);
+                const int kk = mode == ORACLE_W_H15 ? 1 : mode == ORACLE_W_H15K2 ? 2 : mode == ORACLE_W_H15K3 ? 3 : 0;
+                if (kk > 0) {
+                    u = ldexp((double)x < -126.0 ? -126.0 : (double)x, kk);   /* the quantity that is rounded */
                 } else {
                     u = -(double)x; /* boundaries of floor(y + 1/2) sit at half-integers too */
                 }
@@ -277,7 +296,7 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
                     double vmax = 0.0;
                     for (int d = 0; d < D; ++d)
                         if (fabs(vr[d]) > vmax) vmax = fabs(vr[d]);
-                    flip += (mode == ORACLE_W_H15) ? 0.5 * w : w;
+                    flip += kk > 0 ? ldexp(w, -kk) : w;   /* one lattice step is at most w / 2^k */
                     if (vmax > flip_vmax) flip_vmax = vmax;
                     ++flagged;
                 }
@@ -316,7 +335,7 @@ int oracle_attn(const void* q, const void* k, const void* v, int in_dtype, int B
                 int nthreads) {
     if (!q || !k || !v || !O || !LSE) return -1;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || D <= 0 || Hq % Hkv) return -2;
-    if (mode < 0 || mode > 2 || in_dtype < 0 || in_dtype > 1 || tile_n < 0) return -3;
+    if (mode < 0 || mode > 4 || in_dtype < 0 || in_dtype > 1 || tile_n < 0) return -3;
     if (tile_n == 0 && mode != ORACLE_W_EXACT) return -3;
     fesetround(FE_TONEAREST);
     if (!rows) nrows = Sq;

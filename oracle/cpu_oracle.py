@@ -17,7 +17,7 @@ _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "attn_oracle.c"
 _LIB = _HERE / "liboracle.so"
 
-W_EXACT, W_POT, W_H15 = 0, 1, 2
+W_EXACT, W_POT, W_H15, W_H15K2, W_H15K3 = 0, 1, 2, 3, 4
 IN_BF16, IN_FP8_E4M3 = 0, 1
 P_NONE, P_BF16, P_E4M3, P_E5M2 = 0, 1, 2, 3
 

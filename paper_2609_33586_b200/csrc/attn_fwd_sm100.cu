@@ -165,7 +165,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto tmem_O = [&](int t) { return tmem + 256u + 128u * t; };
 
     constexpr uint32_t fmt_ab = FP8 ? kFmtE4M3 : kFmtBF16;
-    constexpr uint32_t fmt_p = FP8 ? (MODE == kExact ? kFmtE4M3 : kFmtE5M2) : kFmtBF16;
+    constexpr uint32_t fmt_p = FP8 ? (PFormat<FP8, MODE>::kE4M3 ? kFmtE4M3 : kFmtE5M2) : kFmtBF16;
     constexpr uint32_t idesc_s = umma_idesc(fmt_ab, fmt_ab, false, false, kTileM, kTileN);
     constexpr uint32_t idesc_pv = umma_idesc(fmt_p, fmt_ab, false, true, kTileM, D);
     constexpr float p_off = static_cast<float>(PFormat<FP8, MODE>::kOffLog2);  // log2 of the P / row-sum scale
@@ -365,7 +365,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_S(t) + lane_base;
         const uint32_t tO = tmem_O(t) + lane_base;
-        const float c_eff = (MODE == kH15) ? 2.0f * p.c : p.c;
+        constexpr int kFam = h15_family_k(MODE);   // h15 family: the map takes the offset times 2^kFam
+        const float c_eff = static_cast<float>(1 << kFam) * p.c;
         int tiles = 0;
         for (int round = 0;; ++round) {
             const int w = item_index(round, cta, n_ctas);
@@ -411,7 +412,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 if (lane == 0) mbar_arrive(bar_scale(t));
                 if (r == 0) ROWMAX_STAMP(t, j, 2);
 
-                // exact: x = s*c - m*c + P offset;  h15: doubled input 2x = s*(2c) - m*(2c);  pot: x = s*c - m*c
+                // exact: x = s*c - m*c + P offset;  h15 family: scaled input 2^K x = s*(2^K c) - m*(2^K c);  pot: x = s*c - m*c
                 RowScale rs;
                 rs.c = make_float2(c_eff, c_eff);
                 const float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
@@ -431,9 +432,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     // 126 octaves below its running maximum; the row minimum (one more three-input pass)
                     // tells, and the common case runs without the per-score clamp.
                     bool clamp = false;
-                    if constexpr (MODE == kH15) {
-                        const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest doubled offset of the row
-                        clamp = __any_sync(0xffffffffu, !(lowest >= -250.0f));
+                    if constexpr (kFam > 0) {
+                        const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest scaled offset of the row
+                        clamp = __any_sync(0xffffffffu, !(lowest >= -125.0f * (1 << kFam)));
                     }
                     if (clamp) {
 #pragma unroll
@@ -554,6 +555,8 @@ static cudaError_t dispatch_mode(int mode, const CUtensorMap& tq, const CUtensor
     switch (mode) {
         case kExact: return launch_ws<D, FP8, kExact>(tq, tk, tv, p, stream);
         case kPot: return launch_ws<D, FP8, kPot>(tq, tk, tv, p, stream);
+        case kH15K2: return launch_ws<D, FP8, kH15K2>(tq, tk, tv, p, stream);
+        case kH15K3: return launch_ws<D, FP8, kH15K3>(tq, tk, tv, p, stream);
         default: return launch_ws<D, FP8, kH15>(tq, tk, tv, p, stream);
     }
 }
@@ -578,7 +581,15 @@ __global__ void weight_map_kernel(const float* __restrict__ x, float* __restrict
         float wi;
         if (mode == kExact) wi = w_exact(xi);
         else if (mode == kPot) wi = w_pot(xi);
-        else wi = w_h15_doubled_pair<0>(make_float2(xi * 2.0f, xi * 2.0f), two22).x;
+        else {
+            // both lanes of the pair function are exercised: even indices take the shift-add lane, odd
+            // indices the multiply-add lane
+            float2 r;
+            if (mode == kH15K2) r = w_h15_doubled_pair<0, true, 2>(make_float2(xi * 4.0f, xi * 4.0f), two22);
+            else if (mode == kH15K3) r = w_h15_doubled_pair<0, true, 3>(make_float2(xi * 8.0f, xi * 8.0f), two22);
+            else r = w_h15_doubled_pair<0, true, 1>(make_float2(xi * 2.0f, xi * 2.0f), two22);
+            wi = (i & 1) ? r.y : r.x;
+        }
         w[i] = wi;
     }
 }

@@ -33,7 +33,10 @@ struct TileCfg {
 // factor, so it cancels in O and is subtracted from LSE.
 template <bool FP8, int MODE>
 struct PFormat {
-    static constexpr int kOffLog2 = FP8 ? (MODE == kExact ? 8 : 15) : 0;
+    // e4m3 (3 fraction bits) for exact mode and for the eighth-octave family member, whose weights
+    // carry 3 fraction bits; e5m2 for pot, h15 and the quarter-octave member (at most 2 fraction bits)
+    static constexpr bool kE4M3 = FP8 && (MODE == kExact || MODE == kH15K3);
+    static constexpr int kOffLog2 = FP8 ? (kE4M3 ? 8 : 15) : 0;
 };
 
 // ---- packed fp32 pairs and small helpers
@@ -158,10 +161,10 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
         if constexpr (MODE == kExact) {
             w.x = w_exact(x.x);  // masked scores are -inf -> weight 0
             w.y = w_exact(x.y);
-        } else if constexpr (MODE == kH15) {
-            // Eq. h15 on the doubled input: clamp at -252, add 2^23 + 2^22 (rounds to the integer n,
-            // ties to even), then (bits << 22) + bias builds (1 + (n mod 2)/2) * 2^(floor(n/2) + kOff).
-            w = w_h15_doubled_pair<kOff, CLAMP>(x, rs.two22);
+        } else if constexpr (h15_family_k(MODE) > 0) {
+            // Eq. h15 on the input scaled by 2^K (K = 1: doubled): clamp, add 2^23 + 2^22 (rounds to the
+            // integer n, ties to even), then (bits << (23 - K)) + bias builds the weight times 2^kOff.
+            w = w_h15_doubled_pair<kOff, CLAMP, h15_family_k(MODE)>(x, rs.two22);
         } else {
             w.x = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.x)) << 23);
             w.y = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.y)) << 23);
@@ -173,18 +176,18 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
         acc[i & 1] = fadd2(acc[i & 1], w);
         if constexpr (!FP8) {
             if constexpr (MODE == kExact) pw[i] = pack_bf16_rn(w.x, w.y);
-            else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: 1 fraction bit
+            else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: at most 3 fraction bits
         } else {
-            if constexpr (MODE == kExact) half16[i] = pack_e4m3x2(w.x, w.y);
-            else half16[i] = pack_f16x2_rn(w.x, w.y);  // lattice weights are exact in fp16 (1 fraction bit)
+            if constexpr (PFormat<FP8, MODE>::kE4M3) half16[i] = pack_e4m3x2(w.x, w.y);
+            else half16[i] = pack_f16x2_rn(w.x, w.y);  // at most 2 fraction bits: exact in fp16
         }
     }
     if constexpr (FP8) {
-        // exact mode: two e4m3 pairs per word.  pot/h15: e5m2 is the upper byte of an fp16 pattern, and a
-        // lattice weight has one fraction bit, so the upper bytes of the four halves are the exact P bytes.
+        // e4m3 P: two converted pairs per word.  e5m2 P: e5m2 is the upper byte of an fp16 pattern, and these
+        // weights have at most two fraction bits, so the upper bytes of the four halves are the exact P bytes.
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-            pw[i] = __byte_perm(half16[2 * i], half16[2 * i + 1], MODE == kExact ? 0x5410 : 0x7531);
+            pw[i] = __byte_perm(half16[2 * i], half16[2 * i + 1], PFormat<FP8, MODE>::kE4M3 ? 0x5410 : 0x7531);
     }
 }
 

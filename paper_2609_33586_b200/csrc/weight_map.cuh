@@ -30,17 +30,22 @@ __device__ __forceinline__ float h15_weight_from_tbits(uint32_t tbits) {
     return __uint_as_float((tbits << 22) + 0x3F800000u);
 }
 __device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_from_tbits(h15_tbits(x2)); }
-// Two weights at once, the form the fused kernel uses: packed fp32 add of the magic constant, then
-// (bits << 22) + bias per lane.  One lane uses the shift-add (ALU pipe), the other the equivalent
-// integer multiply-add t * 2^22 + bias mod 2^32 (FMA pipe), which balances the two pipes; `two22`
-// must hold 1 << 22 and arrives in a register so that the multiply-add is not turned back into a
-// shift.  kOff scales the weight by 2^kOff (an exact exponent shift) for the fp8 P formats.
-// kClamp = false skips the clamp at -252; the caller must know that both inputs are >= -252.
-template <int kOff, bool kClamp = true>
+// Two weights at once, the form the fused kernel uses, for the family member with input steps of
+// 2^-K octaves (K = 1 is Rowmax-H15; K = 2, 3 are the quarter- and eighth-octave members of App. B
+// "Exponential-map ablation": same add, shift by 23 - K).  Input is the offset times 2^K.  Packed fp32
+// add of the magic constant, then (bits << (23 - K)) + bias per lane: the low K bits of n become the
+// top fraction bits and the rest the exponent, i.e. 2^floor(n / 2^K) * (1 + (n mod 2^K) / 2^K).  One
+// lane uses the shift-add (ALU pipe), the other the equivalent integer multiply-add (FMA pipe), which
+// balances the two pipes; `two22` must hold 1 << 22 and arrives in a register so that the
+// multiply-add is not turned back into a shift.  kOff scales the weight by 2^kOff (an exact exponent
+// shift) for the fp8 P formats.  kClamp = false skips the clamp at -126 * 2^K; the caller must know
+// that both inputs are at or above it.
+template <int kOff, bool kClamp = true, int K = 1>
 __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) {
+    static_assert(K >= 1 && K <= 3, "family members k = 1, 2, 3");
     if constexpr (kClamp) {
-        x2.x = fmaxf(x2.x, -252.0f);
-        x2.y = fmaxf(x2.y, -252.0f);
+        x2.x = fmaxf(x2.x, -126.0f * (1 << K));
+        x2.y = fmaxf(x2.y, -126.0f * (1 << K));
     }
     float2 t;
     asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
@@ -49,10 +54,10 @@ __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) 
         "mov.b64 {%0, %1}, rd;\n\t}"
         : "=f"(t.x), "=f"(t.y)
         : "f"(x2.x), "f"(x2.y), "f"(kH15Magic));
-    constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(2 * kOff) << 22);
-    const uint32_t b0 = (__float_as_uint(t.x) << 22) + bias;
+    constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(kOff) << 23);
+    const uint32_t b0 = (__float_as_uint(t.x) << (23 - K)) + bias;
     uint32_t b1;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22), "r"(bias));
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22 >> (K - 1)), "r"(bias));
     return make_float2(__uint_as_float(b0), __uint_as_float(b1));
 }
 

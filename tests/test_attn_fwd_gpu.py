@@ -12,6 +12,7 @@ from parity_util import compare
 pytestmark = pytest.mark.gpu
 
 MODES = [orc.W_EXACT, orc.W_POT, orc.W_H15]
+FAMILY = [orc.W_H15K2, orc.W_H15K3]
 
 
 @pytest.fixture(autouse=True)
@@ -39,6 +40,24 @@ def test_config0_tiny_causal_every_row(mode):
 ], ids=lambda w: w.name)
 def test_small_shapes(wl, mode):
     st = compare(wl, mode)
+    assert st["ok"], st
+
+
+@pytest.mark.parametrize("mode", FAMILY)
+@pytest.mark.parametrize("wl", [
+    Workload("fam_bf16", 2, 4, 2, 300, 428, 128, True, "bf16", 51),
+    Workload("fam_d64", 1, 2, 2, 257, 391, 64, False, "bf16", 52),
+    Workload("fam_fp8", 2, 4, 2, 300, 428, 128, True, "fp8_e4m3", 53),
+], ids=lambda w: w.name)
+def test_h15_family_members_small_shapes(wl, mode):
+    st = compare(wl, mode)
+    assert st["ok"], st
+
+
+@pytest.mark.parametrize("mode", FAMILY)
+def test_h15_family_members_full_size_8k_fp8(mode):
+    wl = WORKLOADS[2]
+    st = compare(wl, mode, rows=_sample_rows(wl.Sq, 256))
     assert st["ok"], st
 
 

@@ -162,6 +162,10 @@ def _numpy_online(q, k, v, causal, scale, mode, tile_n, order=1, tau=0.0, kmax=2
             return np.exp2(x)
         if mode == orc.W_POT:
             return np.exp2(-np.minimum(kmax, np.floor(-x + 0.5)))
+        if mode in (orc.W_H15K2, orc.W_H15K3):
+            st = 4.0 if mode == orc.W_H15K2 else 8.0
+            q = np.rint(st * np.maximum(x, -126.0)) / st
+            return np.exp2(np.floor(q)) * (1.0 + q - np.floor(q))
         n = np.rint(2.0 * np.maximum(x, -126.0))
         return np.where(n % 2 == 0, 1.0, 1.5) * np.exp2(np.floor(n / 2.0))
 
@@ -191,7 +195,7 @@ def _numpy_online(q, k, v, causal, scale, mode, tile_n, order=1, tau=0.0, kmax=2
     return O, L
 
 
-@pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_POT, orc.W_H15])
+@pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_POT, orc.W_H15, orc.W_H15K2, orc.W_H15K3])
 @pytest.mark.parametrize("tile_n,order,tau", [(16, 1, 0.0), (16, -1, 0.0), (8, 1, 3.0)])
 def test_online_matches_independent_numpy_coding(mode, tile_n, order, tau):
     wl = TINY_X

@@ -112,6 +112,43 @@ def test_h15_equals_add_and_shift_bit_construction():
         assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
 
 
+# ---- the family H15 belongs to: S(Q_{2^-k}(x)), k = 2, 3 (App. B "Exponential-map ablation") ----
+
+def _schraudolph(q):
+    return np.exp2(np.floor(q)) * (1.0 + q - np.floor(q))
+
+
+@pytest.mark.parametrize("k,mode", [(2, orc.W_H15K2), (3, orc.W_H15K3)])
+def test_h15_family_equals_schraudolph_on_rounded_input_and_the_shift_construction(k, mode):
+    x = inputs.paper_bit_test_set()
+    q = np.rint(x.astype(np.float64) * 2 ** k) / 2 ** k           # independent coding of Q_{2^-k}
+    got = orc.weight_map(x, mode)
+    assert np.array_equal(got, _schraudolph(q))
+    # the add-and-shift pattern with 2^k x and a left shift by 23 - k
+    magic = np.array([0x4B400000], dtype=np.uint32).view(np.float32)[0]
+    t = (np.maximum(x * np.float32(2 ** k), np.float32(-126 * 2 ** k)).astype(np.float32) + magic).astype(np.float32)
+    bits = (t.view(np.uint32) << np.uint32(23 - k)) + np.uint32(0x3F800000)
+    assert np.array_equal(got.astype(np.float32).view(np.uint32), bits)
+
+
+def test_h15_family_k1_is_h15_and_envelopes_shrink_with_k():
+    x = inputs.paper_bit_test_set()
+    assert np.array_equal(orc.weight_map(x, orc.W_H15), _schraudolph(np.rint(2.0 * x.astype(np.float64)) / 2.0))
+    interp = 0.08607133205593432       # max of log2(1 + f) - f, attained at f = 1/ln 2 - 1
+    for k, mode in ((2, orc.W_H15K2), (3, orc.W_H15K3)):
+        w = orc.weight_map(x, mode)
+        eps = np.log2(w) - x.astype(np.float64)
+        half_step = 2.0 ** -(k + 1)   # |q - x| <= half an input step; log2 S(q) - q lies in [0, interp]
+        assert eps.min() >= -half_step - 1e-12 and eps.max() <= interp + half_step + 1e-12
+        xs = np.sort(inputs.weight_map_sweep())
+        ws = orc.weight_map(xs, mode)
+        assert np.all(np.diff(ws) >= 0)
+        assert orc.weight_map(np.array([0.0, -126.0, -200.0, -np.inf], np.float32), mode).tolist() == \
+            [1.0, 2.0 ** -126, 2.0 ** -126, 2.0 ** -126]
+        frac_bits = np.unique(np.frexp(w)[0] * 2 ** (k + 1))       # mantissa in [0.5,1) has k fraction bits
+        assert np.all(frac_bits == np.round(frac_bits))
+
+
 def test_h15_minus_infinity_is_the_clamp_value():
     w = orc.weight_map(np.array([-np.inf, -150.0, -126.0], np.float32), orc.W_H15)
     assert np.all(w == 2.0 ** -126)

@@ -15,7 +15,7 @@ def _gpu_map(x, mode):
     return binding.weight_map(xt, mode).cpu().numpy()
 
 
-@pytest.mark.parametrize("mode", [orc.W_H15, orc.W_POT])
+@pytest.mark.parametrize("mode", [orc.W_H15, orc.W_POT, orc.W_H15K2, orc.W_H15K3])
 def test_rounding_maps_are_bit_exact_on_the_sweep(mode):
     for x in (inputs.weight_map_sweep(), inputs.paper_bit_test_set()):
         if mode == orc.W_POT:
