@@ -414,8 +414,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
                 // exact: x = s*c - m*c + P offset;  h15 family: scaled input 2^K x = s*(2^K c) - m*(2^K c);  pot: x = s*c - m*c
                 RowScale rs;
-                rs.c = make_float2(c_eff, c_eff);
-                const float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
+                float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
+                float c_row = c_eff;
+                if constexpr (MODE == kPot) {   // pot works on y = -x = m*c - s*c
+                    nmc = -nmc;
+                    c_row = -c_eff;
+                }
+                rs.c = make_float2(c_row, c_row);
                 rs.nmc = make_float2(nmc, nmc);
                 rs.two22 = p.two22;
                 float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};

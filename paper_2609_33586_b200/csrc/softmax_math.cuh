@@ -166,8 +166,9 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             // integer n, ties to even), then (bits << (23 - K)) + bias builds the weight times 2^kOff.
             w = w_h15_doubled_pair<kOff, CLAMP, h15_family_k(MODE)>(x, rs.two22);
         } else {
-            w.x = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.x)) << 23);
-            w.y = __uint_as_float(static_cast<uint32_t>(127 + kOff - pot_index(x.y)) << 23);
+            // rs.c and rs.nmc carry the opposite sign in pot mode: x holds y = -(offset) >= 0
+            w.x = pot_weight_from_y<kOff>(x.x);
+            w.y = pot_weight_from_y<kOff>(x.y);
         }
         if constexpr (MODE != kExact && MASKED) {
             if (2 * i >= limit) w.x = 0.f;

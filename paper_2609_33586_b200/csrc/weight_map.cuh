@@ -64,15 +64,25 @@ __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) 
 // ---- Rowmax-PoT (Eq. rowmax-pot): d = min{K_max, floor(y + 1/2)}, y = -x, w = 2^-d.
 // floor(y + 1/2) without double rounding: one round-DOWN add of 2^22 + 64.5 leaves
 // 2^22 + floor(2 (y + 64.5)) / 2 exactly, whose integer part is floor(y + 1/2) + 64.
-__device__ __forceinline__ int pot_index(float x) {
-    float y = fminf(fmaxf(-x, -64.0f), 64.0f);
-    float t = __fadd_rd(y, 4194368.5f);
-    int twice = static_cast<int>(__float_as_uint(t) - 0x4A800000u);  // 2 * (t - 2^22)
-    int d = (twice >> 1) - 64;
-    return min(d, kPotKmax);
+// Capping y at K_max + 1/4 first makes the min{K_max, .} implicit (floor(y + 1/2) = K_max for every
+// y in [K_max - 1/2, K_max + 1/2)) and keeps huge and infinite y in range.  y >= -64 is required
+// (offsets above the anchor occur only with a deferred rescale, whose threshold is at most 32).
+constexpr float kPotMagic = 4194368.5f;        // 2^22 + 64.5, bit pattern 0x4A800081
+constexpr uint32_t kPotMagicBase = 0x4A800000u;  // bit pattern of 2^22
+__device__ __forceinline__ uint32_t pot_tbits(float y) {
+    return __float_as_uint(__fadd_rd(fminf(y, static_cast<float>(kPotKmax) + 0.25f), kPotMagic));
 }
-__device__ __forceinline__ float w_pot(float x) {
-    return __uint_as_float(static_cast<uint32_t>(127 - pot_index(x)) << 23);
+__device__ __forceinline__ int pot_index_from_y(float y) {
+    return static_cast<int>((pot_tbits(y) - kPotMagicBase) >> 1) - 64;   // (2 (t - 2^22)) / 2 - 64
 }
+__device__ __forceinline__ int pot_index(float x) { return pot_index_from_y(-x); }
+// fp32 pattern of 2^(kOff - d): exponent field 127 + kOff - d = (191 + kOff) - (d + 64), and d + 64 is
+// the t pattern without its lowest bit, shifted right by one: ((tbits & ~1) << 22) puts it at bit 23
+// (the bits of 2^22's own pattern fall off the top).
+template <int kOff>
+__device__ __forceinline__ float pot_weight_from_y(float y) {
+    return __uint_as_float((static_cast<uint32_t>(191 + kOff) << 23) - ((pot_tbits(y) & ~1u) << 22));
+}
+__device__ __forceinline__ float w_pot(float x) { return pot_weight_from_y<0>(-x); }
 
 }  // namespace rowmax
