@@ -263,6 +263,38 @@ def speedup_rounds(run: DeviceRun, steps: int, device, rounds: int = 3):
             "speedup_pct_per_round": per_round, "windows_per_mode": rounds, "calls_per_window": steps}
 
 
+def energy_leg(run: DeviceRun, index: int, seconds: float):
+    """Board energy per forward, the paper's way (App. B "Energy"): a loop of forwards in chunks of 50
+    calls, each followed by a synchronisation, while NVML board power is sampled; energy = mean power
+    x loop time / forwards completed, no idle power subtracted.  One loop per mode, exact then h15."""
+    out = {}
+    for name in ("exact", "h15"):
+        mode = MODE_IDS[name]
+        for _ in range(30):
+            run.step(mode)
+        torch.cuda.synchronize()
+        with ClockSampler(index) as smp:
+            t0 = time.perf_counter()
+            n = 0
+            while time.perf_counter() - t0 < seconds:
+                for _ in range(50):
+                    run.step(mode)
+                torch.cuda.synchronize()
+                n += 50
+            t1 = time.perf_counter()
+        powers = [s[1] for s in smp.samples]
+        if not powers or n == 0:
+            return None
+        skip = min(len(powers) // 10, 50)          # drop the start-up ramp
+        mean_w = statistics.mean(powers[skip:])
+        sm = statistics.median(s[0] for s in smp.samples)
+        out[name] = {"mj_per_forward": 1e3 * mean_w * (t1 - t0) / n, "mean_power_w": mean_w, "forwards": n,
+                     "loop_s": t1 - t0, "ms_per_forward": 1e3 * (t1 - t0) / n, "sm_mhz_median": sm}
+    out["h15_energy_change_pct"] = 100.0 * (out["h15"]["mj_per_forward"] / out["exact"]["mj_per_forward"] - 1.0)
+    out["workload"] = run.wl.name
+    return out
+
+
 def e2e_leg(run: DeviceRun, steps: int, warmup: int):
     """Same step from pinned host buffers: H2D of q, k, v, the kernel, D2H of O and LSE, all on the
     launching stream and inside the timed region."""
@@ -331,6 +363,7 @@ def run_ours(args):
         sp = speedup_rounds(run, args.steps, device)
         sp_nc = speedup_rounds(twin, args.steps, device)
     clocks = clk.summary()
+    energy = energy_leg(run, local_rank, args.energy_seconds) if (world == 1 and args.energy_seconds > 0) else None
     ms_e2e, h2d, d2h = e2e_leg(run, max(3, args.steps // 4), args.warmup)
     ms_e2e = max_over_ranks(ms_e2e, device)
     status = binding.device_status()
@@ -359,6 +392,8 @@ def run_ours(args):
             "noncausal_8k_fp8": dict(sp_nc, h15_tflops=tf(TWIN, sp_nc["h15_ms"]), exact_tflops=tf(TWIN, sp_nc["exact_ms"])),
         },
     }
+    if energy is not None:
+        line["energy"] = energy
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg(wl, inp)
@@ -375,6 +410,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
+    ap.add_argument("--energy-seconds", type=float, default=4.0,
+                    help="length of the energy loop per mode at N=1 (0 = skip)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -532,23 +532,24 @@ static cudaError_t launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const
                              const AttnParams& p, cudaStream_t stream) {
     using W = WsCfg<D, FP8>;
     auto kern = attn_fwd_ws_kernel<D, FP8, MODE>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, W::kSmemBytes);
+    // per-device launch set-up: the shared-memory opt-in of this instance and the SM count
+    static bool configured[64] = {};
+    static int sm_counts[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, W::kSmemBytes);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_counts[dev], cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
+    const int sm_count = sm_counts[dev];
     const long long n_pairs = (p.Sq + 2 * kTileM - 1) / (2 * kTileM);
     const long long items = n_pairs * p.Hq * p.B;
     if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
     // persistent CTAs: one per SM (shared memory and TMEM allow no more), each walking its share of the items
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-    }
     const unsigned blocks = static_cast<unsigned>(items < sm_count ? items : sm_count);
     kern<<<blocks, 512, W::kSmemBytes, stream>>>(tq, tk, tv, p);
     return cudaGetLastError();
