@@ -36,30 +36,40 @@ def run_cuda(wl: Workload, inp: Inputs, mode: int, device="cuda:0", tau=None):
     return o, lse
 
 
-def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None):
+def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None, model_p_storage=False):
     dt = orc.IN_BF16 if wl.in_dtype == "bf16" else orc.IN_FP8_E4M3
     sch = binding.get_schedule(wl.D, dt, mode, wl.causal)
     assert sch["rescale_tau"] == 0.0
     if tau is not None:
         sch["rescale_tau"] = tau
     tile = 0 if mode == orc.W_EXACT else sch["tile_n"]   # exact mode: the whole-row definition
+    p_kw = {}
+    if model_p_storage and sch["p_format"] == binding.P_E4M3:
+        # diagnostic reference: the online loop with P rounded to the kernel's e4m3 storage format
+        tile = sch["tile_n"]
+        p_kw = {"p_round": orc.P_E4M3, "p_off": sch["p_offset_log2"]}
     return orc.attn(storage_bits(inp.q), storage_bits(inp.k), storage_bits(inp.v), in_dtype=dt,
                     causal=wl.causal, softmax_scale=wl.softmax_scale, mode=mode, tile_n=tile,
                     kv_order=sch["kv_order"], tau=sch["rescale_tau"], kmax=sch["pot_kmax"],
                     q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale,
-                    tie_eps=TIE_EPS if mode != orc.W_EXACT else 0.0, rows=rows)
+                    tie_eps=TIE_EPS if mode != orc.W_EXACT else 0.0, rows=rows, **p_kw)
 
 
 def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, device="cuda:0",
-            allow_output_rounding: bool = False, tau=None):
+            allow_output_rounding: bool = False, tau=None, model_p_storage: bool = False):
     """Returns a dict of error statistics; `ok` says whether every gate holds.
 
+    `model_p_storage`: where the kernel stores P in e4m3 (exact mode, and the eighth-octave family
+    member, on fp8 inputs) the reference is the oracle's online loop with P rounded to that format.
+    Used for inputs with peaked rows, where two or three weights carry a row and their 3-fraction-bit
+    rounding shows in O far beyond 5e-2 against the unrounded reference; the standard workloads are
+    compared with the unrounded reference.
     `allow_output_rounding` adds half a bf16 ulp of the reference value to the per-row tolerance: O
     is stored in bf16, and for outputs of magnitude 2 and above that rounding alone is 0.008 and
     more.  The standard workloads (N(0,1) values, averaged) do not need it."""
     inp = inp or make_inputs(wl)
     o, lse = run_cuda(wl, inp, mode, device, tau)
-    ref = run_oracle(wl, inp, mode, rows, tau)
+    ref = run_oracle(wl, inp, mode, rows, tau, model_p_storage)
     o = o.float().cpu().numpy().transpose(0, 2, 1, 3).astype(np.float64)   # (B,Hq,Sq,D)
     lse = lse.cpu().numpy().astype(np.float64)
     if rows is not None:
@@ -75,7 +85,8 @@ def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, devic
     if allow_output_rounding:
         allowed = allowed + np.abs(ref["O"]).max(axis=-1) * 2.0 ** -8
     inf_both = np.isneginf(lse) & np.isneginf(ref["LSE"])
-    err_l = np.where(inf_both, 0.0, np.abs(lse - ref["LSE"]))
+    with np.errstate(invalid="ignore"):
+        err_l = np.where(inf_both, 0.0, np.abs(lse - ref["LSE"]))
     err_l = np.where(np.isnan(err_l), np.inf, err_l)
     allowed_l = tol["lse"] + ref["widen_lse"]
     clean = ref["nflag"] == 0

@@ -61,6 +61,37 @@ def test_h15_family_members_full_size_8k_fp8(mode):
     assert st["ok"], st
 
 
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        dtype = "fp8_e4m3" if rng.random() < 0.4 else "bf16"
+        D = 128 if dtype == "fp8_e4m3" or rng.random() < 0.6 else 64
+        hkv = int(rng.integers(1, 4))
+        g = int(rng.choice([1, 2, 4]))
+        B = int(rng.integers(1, 4))
+        Sq = int(rng.integers(1, 700))
+        Sk = int(rng.integers(1, 900))
+        causal = bool(rng.random() < 0.6)
+        out.append(Workload(f"fuzz{i}", B, hkv * g, hkv, Sq, Sk, D, causal, dtype, 100 + i, peaked_keys=bool(rng.random() < 0.3)))
+    return out
+
+
+@pytest.mark.parametrize("wl", _random_shapes(24, 7), ids=lambda w: f"{w.name}-{w.in_dtype}-B{w.B}H{w.Hq}/{w.Hkv}-{w.Sq}x{w.Sk}-D{w.D}-{'c' if w.causal else 'n'}")
+def test_random_shapes_all_modes(wl):
+    # ragged lengths, Sq != Sk in both directions, grouped heads, more work items than CTAs or fewer
+    for mode in MODES + FAMILY:
+        st = compare(wl, mode, model_p_storage=True)
+        assert st["ok"], (mode, st)
+
+
+def test_many_work_items_per_cta():
+    # 4 x 40 heads x 3 tile pairs = 480 items on 148 persistent CTAs: several rounds of the snake per CTA
+    wl = Workload("many", 4, 40, 8, 700, 700, 64, True, "bf16", 61)
+    st = compare(wl, orc.W_H15, rows=_sample_rows(wl.Sq, 7))
+    assert st["ok"], st
+
+
 @pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_H15])
 def test_config1_gqa_peaked_rows(mode):
     wl = WORKLOADS[1]
