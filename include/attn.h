@@ -11,6 +11,9 @@
  *   h15   : (1 + (n mod 2)/2) 2^floor(n/2), n = RNE(2x)   Rowmax-H15, Eq. m-h15 (Sec. 5.2) / Eq. h15 (App. B.1)
  *   h15k2, h15k3 : 2^floor(q) (1 + q - floor(q)), q = RNE(2^k x)/2^k, k = 2, 3   the family H15 belongs to
  *           (k = 1), App. B "Exponential-map ablation": same add-and-shift with 2^k x and a shift by 23 - k
+ *   exact_poly : 2^x as in exact, but every fourth pair of scores evaluated by floor + cubic + exponent insert
+ *           instead of the special-function unit (relative error <= 1.1e-4): the partial emulation of the
+ *           paper's baseline kernel, a stronger control than plain exact (App. B "FA4's own parameter space")
  * and x is the score's base-two offset from the running row maximum of the online-softmax loop
  * over key tiles (Sec. 5.2, App. B.1): x = s*c - m*c with c = softmax_scale*q_descale*k_descale*log2(e).
  * In pot and h15 mode the result depends on the key-tile schedule, which attn_get_schedule reports.
@@ -33,7 +36,8 @@ extern "C" {
 #endif
 
 enum { ATTN_W_EXACT = 0, ATTN_W_POT = 1, ATTN_W_H15 = 2,
-       ATTN_W_H15K2 = 3, ATTN_W_H15K3 = 4 };   /* quarter- and eighth-octave members of the H15 family */
+       ATTN_W_H15K2 = 3, ATTN_W_H15K3 = 4,     /* quarter- and eighth-octave members of the H15 family */
+       ATTN_W_EXACT_POLY = 5 };               /* exact, a quarter of the 2^x evaluated by a cubic on the FMA pipe */
 enum { ATTN_IN_BF16 = 0, ATTN_IN_FP8_E4M3 = 1 };
 /* format of the probability tile P fed to the P.V contraction, as reported by attn_get_schedule */
 enum { ATTN_P_BF16 = 0, ATTN_P_E4M3 = 1, ATTN_P_E5M2 = 2 };
@@ -63,7 +67,7 @@ enum {
  *                corner); a row that sees no key gets O = 0 and LSE = -inf
  *   Hq, Hkv      query head h reads key/value head h / (Hq / Hkv)
  *   softmax_scale  multiplies q.k before the softmax (natural-exponent units)
- *   weight_mode  ATTN_W_EXACT / ATTN_W_POT / ATTN_W_H15 / ATTN_W_H15K2 / ATTN_W_H15K3
+ *   weight_mode  ATTN_W_EXACT / ATTN_W_POT / ATTN_W_H15 / ATTN_W_H15K2 / ATTN_W_H15K3 / ATTN_W_EXACT_POLY
  *   q/k/v_descale  per-tensor factors of the fp8 inputs (value = stored * descale); ignored for bf16
  *
  * All tensors are contiguous; q, k, v, o must be 16-byte aligned.  In pot/h15 mode LSE is the log

@@ -11,10 +11,11 @@ from pathlib import Path
 
 import torch
 
-W_EXACT, W_POT, W_H15, W_H15K2, W_H15K3 = 0, 1, 2, 3, 4
+W_EXACT, W_POT, W_H15, W_H15K2, W_H15K3, W_EXACT_POLY = 0, 1, 2, 3, 4, 5
 IN_BF16, IN_FP8_E4M3 = 0, 1
 P_BF16, P_E4M3, P_E5M2 = 0, 1, 2
-MODES = {"exact": W_EXACT, "pot": W_POT, "h15": W_H15, "h15k2": W_H15K2, "h15k3": W_H15K3}
+MODES = {"exact": W_EXACT, "pot": W_POT, "h15": W_H15, "h15k2": W_H15K2, "h15k3": W_H15K3,
+         "exact_poly": W_EXACT_POLY}
 
 _LIB_PATH = Path(__file__).resolve().parent / "libattn_b200.so"
 _lib = None

@@ -116,7 +116,7 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
                  int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
                  float k_descale, float v_descale, float rescale_tau, void* stream) {
     if (!q || !k || !v || !o) return ATTN_ERR_NULLPTR;
-    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15K3) return ATTN_ERR_BAD_ENUM;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
     if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return ATTN_ERR_BAD_SHAPE;
     if (D != 64 && D != 128) return ATTN_ERR_BAD_SHAPE;
@@ -177,7 +177,7 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, i
 int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* stream) {
     if (n == 0) return ATTN_OK;
     if (!x || !w) return ATTN_ERR_NULLPTR;
-    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15K3) return ATTN_ERR_BAD_ENUM;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
     cudaError_t e = rowmax::launch_weight_map(x, w, n, weight_mode, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(e);
@@ -192,14 +192,14 @@ int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* til
     (void)causal;
     if (D != 64 && D != 128) return ATTN_ERR_BAD_SHAPE;
     if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
-    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_H15K3) return ATTN_ERR_BAD_ENUM;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
     const bool fp8 = in_dtype == ATTN_IN_FP8_E4M3;
     if (tile_m) *tile_m = rowmax::kTileM;
     if (tile_n) *tile_n = rowmax::kTileN;
     if (kv_order) *kv_order = +1;
     if (rescale_tau) *rescale_tau = 0.0f;
     if (pot_kmax) *pot_kmax = 20;
-    const bool e4m3 = weight_mode == ATTN_W_EXACT || weight_mode == ATTN_W_H15K3;
+    const bool e4m3 = weight_mode == ATTN_W_EXACT || weight_mode == ATTN_W_EXACT_POLY || weight_mode == ATTN_W_H15K3;
     if (p_format) *p_format = !fp8 ? ATTN_P_BF16 : (e4m3 ? ATTN_P_E4M3 : ATTN_P_E5M2);
     if (p_offset_log2) *p_offset_log2 = !fp8 ? 0 : (e4m3 ? 8 : 15);
     return ATTN_OK;

@@ -414,7 +414,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
                 // exact: x = s*c - m*c + P offset;  h15 family: scaled input 2^K x = s*(2^K c) - m*(2^K c);  pot: x = s*c - m*c
                 RowScale rs;
-                float nmc = (MODE == kExact ? p_off : 0.0f) - m_use * c_eff;
+                float nmc = (is_exact_like(MODE) ? p_off : 0.0f) - m_use * c_eff;
                 float c_row = c_eff;
                 if constexpr (MODE == kPot) {   // pot works on y = -x = m*c - s*c
                     nmc = -nmc;
@@ -563,6 +563,7 @@ static cudaError_t dispatch_mode(int mode, const CUtensorMap& tq, const CUtensor
         case kPot: return launch_ws<D, FP8, kPot>(tq, tk, tv, p, stream);
         case kH15K2: return launch_ws<D, FP8, kH15K2>(tq, tk, tv, p, stream);
         case kH15K3: return launch_ws<D, FP8, kH15K3>(tq, tk, tv, p, stream);
+        case kExactPoly: return launch_ws<D, FP8, kExactPoly>(tq, tk, tv, p, stream);
         default: return launch_ws<D, FP8, kH15>(tq, tk, tv, p, stream);
     }
 }
@@ -586,6 +587,7 @@ __global__ void weight_map_kernel(const float* __restrict__ x, float* __restrict
         const float xi = x[i];
         float wi;
         if (mode == kExact) wi = w_exact(xi);
+        else if (mode == kExactPoly) wi = w_exact_poly3(xi);
         else if (mode == kPot) wi = w_pot(xi);
         else {
             // both lanes of the pair function are exercised: even indices take the shift-add lane, odd

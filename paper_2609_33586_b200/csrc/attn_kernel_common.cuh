@@ -8,7 +8,9 @@ namespace rowmax {
 constexpr int kTileM = 128;  // query rows per tile
 constexpr int kTileN = 128;  // keys per tile
 
-enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4 };
+enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4, kExactPoly = 5 };
+// modes whose weight is 2^x itself (with the P offset folded into x)
+__host__ __device__ constexpr bool is_exact_like(int mode) { return mode == kExact || mode == kExactPoly; }
 // input-rounding exponent of the h15 family member: steps of 2^-k octaves (0: not a family member)
 __host__ __device__ constexpr int h15_family_k(int mode) {
     return mode == kH15 ? 1 : mode == kH15K2 ? 2 : mode == kH15K3 ? 3 : 0;

@@ -35,7 +35,7 @@ template <bool FP8, int MODE>
 struct PFormat {
     // e4m3 (3 fraction bits) for exact mode and for the eighth-octave family member, whose weights
     // carry 3 fraction bits; e5m2 for pot, h15 and the quarter-octave member (at most 2 fraction bits)
-    static constexpr bool kE4M3 = FP8 && (MODE == kExact || MODE == kH15K3);
+    static constexpr bool kE4M3 = FP8 && (is_exact_like(MODE) || MODE == kH15K3);
     static constexpr int kOffLog2 = FP8 ? (kE4M3 ? 8 : 15) : 0;
 };
 
@@ -158,7 +158,16 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
         const float2 sv = make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
         float2 x = ffma2(sv, rs.c, rs.nmc);
         float2 w;
-        if constexpr (MODE == kExact) {
+        if constexpr (MODE == kExactPoly && !MASKED) {
+            // every fourth pair (25 % of the scores) takes the polynomial route, the rest the hardware ex2
+            if (i % 4 == 3) {
+                w.x = w_exact_poly3(x.x);
+                w.y = w_exact_poly3(x.y);
+            } else {
+                w.x = w_exact(x.x);
+                w.y = w_exact(x.y);
+            }
+        } else if constexpr (is_exact_like(MODE)) {
             w.x = w_exact(x.x);  // masked scores are -inf -> weight 0
             w.y = w_exact(x.y);
         } else if constexpr (h15_family_k(MODE) > 0) {
@@ -170,13 +179,13 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             w.x = pot_weight_from_y<kOff>(x.x);
             w.y = pot_weight_from_y<kOff>(x.y);
         }
-        if constexpr (MODE != kExact && MASKED) {
+        if constexpr (!is_exact_like(MODE) && MASKED) {
             if (2 * i >= limit) w.x = 0.f;
             if (2 * i + 1 >= limit) w.y = 0.f;
         }
         acc[i & 1] = fadd2(acc[i & 1], w);
         if constexpr (!FP8) {
-            if constexpr (MODE == kExact) pw[i] = pack_bf16_rn(w.x, w.y);
+            if constexpr (is_exact_like(MODE)) pw[i] = pack_bf16_rn(w.x, w.y);
             else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: at most 3 fraction bits
         } else {
             if constexpr (PFormat<FP8, MODE>::kE4M3) half16[i] = pack_e4m3x2(w.x, w.y);

@@ -14,6 +14,20 @@ __device__ __forceinline__ float w_exact(float x) {
     return y;
 }
 
+// ---- exact, emulated on the FMA and ALU pipes (the partial emulation the paper's baseline kernel uses to
+// take load off the special-function unit, Sec. 1 and App. B "FA4's own parameter space"): floor(x) by a
+// round-down add of 2^23 + 2^22, a cubic for 2^f on the fraction f in [0,1), and floor(x) added to the
+// exponent field.  The cubic is this build's own fit: it interpolates 2^0 and 2^1 (so the map is continuous
+// across octaves) and minimises the largest relative error on [0,1], which is 1.03e-4.
+// Valid for -126 <= x < 127; smaller inputs are clamped, so the result is never exactly zero.
+__device__ __forceinline__ float w_exact_poly3(float x) {
+    x = fmaxf(x, -126.0f);
+    const float t = __fadd_rd(x, 12582912.0f);   // 2^23 + 2^22 + floor(x), exact
+    const float f = x - (t - 12582912.0f);       // fraction in [0,1)
+    const float p = fmaf(fmaf(fmaf(0.07826797f, f, 0.22630768f), f, 0.69542432f), f, 1.0f);   // 2^f in [1,2]
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
 // ---- Rowmax-H15 (Eq. h15; construction of App. B.1 "Implementation").
 // Input is the DOUBLED offset 2x.  After the clamp at -252, adding 2^23 + 2^22 as an fp32 value
 // rounds 2x to the nearest integer n (ties to even) and leaves 0x4B400000 + n in the bit pattern.

@@ -27,7 +27,7 @@ def test_host_only_entry_points_work_without_a_gpu():
     assert binding.version().startswith("rowmax-attn-b200")
     assert binding.status_string(0) == "ok" and "shape" in binding.status_string(-2)
     for in_dtype, mode, fmt, off in ((0, 2, binding.P_BF16, 0), (1, 0, binding.P_E4M3, 8), (1, 2, binding.P_E5M2, 15),
-                                     (1, 3, binding.P_E5M2, 15), (1, 4, binding.P_E4M3, 8)):
+                                     (1, 3, binding.P_E5M2, 15), (1, 4, binding.P_E4M3, 8), (1, 5, binding.P_E4M3, 8)):
         s = binding.get_schedule(128, in_dtype, mode, True)
         assert (s["tile_m"], s["tile_n"], s["kv_order"], s["rescale_tau"], s["pot_kmax"]) == (128, 128, 1, 0.0, 20)
         assert (s["p_format"], s["p_offset_log2"]) == (fmt, off)

@@ -13,6 +13,7 @@ pytestmark = pytest.mark.gpu
 
 MODES = [orc.W_EXACT, orc.W_POT, orc.W_H15]
 FAMILY = [orc.W_H15K2, orc.W_H15K3]
+EXACT_POLY = binding.W_EXACT_POLY
 
 
 @pytest.fixture(autouse=True)
@@ -54,6 +55,23 @@ def test_h15_family_members_small_shapes(wl, mode):
     assert st["ok"], st
 
 
+@pytest.mark.parametrize("wl", [
+    Workload("poly_bf16", 2, 4, 2, 300, 428, 128, True, "bf16", 54),
+    Workload("poly_d64", 1, 2, 2, 257, 391, 64, False, "bf16", 55),
+    Workload("poly_fp8", 2, 4, 2, 300, 428, 128, True, "fp8_e4m3", 56),
+    WORKLOADS[0],
+], ids=lambda w: w.name)
+def test_partly_emulated_exact_mode_meets_the_exact_tolerances(wl):
+    st = compare(wl, EXACT_POLY)
+    assert st["ok"], st
+
+
+def test_partly_emulated_exact_mode_full_size_8k_fp8():
+    wl = WORKLOADS[2]
+    st = compare(wl, EXACT_POLY, rows=_sample_rows(wl.Sq, 256))
+    assert st["ok"], st
+
+
 @pytest.mark.parametrize("mode", FAMILY)
 def test_h15_family_members_full_size_8k_fp8(mode):
     wl = WORKLOADS[2]
@@ -80,7 +98,7 @@ def _random_shapes(n, seed):
 @pytest.mark.parametrize("wl", _random_shapes(24, 7), ids=lambda w: f"{w.name}-{w.in_dtype}-B{w.B}H{w.Hq}/{w.Hkv}-{w.Sq}x{w.Sk}-D{w.D}-{'c' if w.causal else 'n'}")
 def test_random_shapes_all_modes(wl):
     # ragged lengths, Sq != Sk in both directions, grouped heads, more work items than CTAs or fewer
-    for mode in MODES + FAMILY:
+    for mode in MODES + FAMILY + [EXACT_POLY]:
         st = compare(wl, mode, model_p_storage=True)
         assert st["ok"], (mode, st)
 
@@ -212,7 +230,7 @@ def test_argument_errors_are_reported_without_launching():
                               0, 0, 1.0, 1.0, 1.0, None)
     assert rc == -1
     rc = binding.attn_fwd_raw(q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128,
-                              128, 1, 0.1, 5, 0, 1.0, 1.0, 1.0, None)
+                              128, 1, 0.1, 9, 0, 1.0, 1.0, 1.0, None)
     assert rc == -3
     rc = binding.attn_fwd_raw(q.data_ptr() + 2, q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 64, 64,
                               128, 1, 0.1, 0, 0, 1.0, 1.0, 1.0, None)

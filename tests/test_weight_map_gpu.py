@@ -44,6 +44,17 @@ def test_exact_map_within_two_ulp_and_flushes_subnormals():
     assert _gpu_map(np.array([-np.inf], np.float32), orc.W_EXACT)[0] == 0.0
 
 
+def test_emulated_exact_map_is_within_its_stated_error():
+    x = inputs.weight_map_sweep()
+    x = x[np.isfinite(x) & (x >= -126.0)]
+    got = _gpu_map(x, binding.W_EXACT_POLY).astype(np.float64)
+    want = orc.weight_map(x, orc.W_EXACT)
+    assert np.max(np.abs(got / want - 1.0)) <= 1.1e-4
+    assert np.all(np.diff(got[np.argsort(x, kind="stable")]) >= 0)          # monotone, continuous across octaves
+    ints = np.arange(-126, 17, dtype=np.float32)
+    assert np.array_equal(_gpu_map(ints, binding.W_EXACT_POLY), np.exp2(ints.astype(np.float64)).astype(np.float32))
+
+
 def test_in_place_and_empty():
     x = torch.tensor([-1.5, 0.0], device="cuda")
     binding.weight_map(x, orc.W_H15, out=x)
