@@ -37,9 +37,20 @@ struct WsCfg {
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
 };
 
-__device__ __forceinline__ void reg_dec_48() { asm volatile("setmaxnreg.dec.sync.aligned.u32 48;"); }
-__device__ __forceinline__ void reg_dec_80() { asm volatile("setmaxnreg.dec.sync.aligned.u32 80;"); }
-__device__ __forceinline__ void reg_inc_192() { asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); }
+// Register split of the 512 threads x 128 registers the CTA is launched with (setmaxnreg can only
+// redistribute that allocation; a larger total would make the increase wait for ever): softmax /
+// correction / MMA+TMA warpgroups.  The lattice modes (two weight variants in the loop, packed P words
+// kept alive) measured faster with more softmax registers, the exact modes with the other split.
+template <int MODE>
+struct RegCfg {
+    static constexpr bool kWide = !is_exact_like(MODE);
+    static constexpr int kSoftmax = kWide ? 208 : 192;
+    static constexpr int kCorr = kWide ? 56 : 80;
+    static constexpr int kMma = kWide ? 40 : 48;
+    static_assert(256 * kSoftmax + 128 * kCorr + 128 * kMma <= 512 * 128, "setmaxnreg targets exceed the launch allocation");
+};
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // Optional cycle stamps (compiled in only with -DROWMAX_TRACE): one representative thread per role of
 // one chosen CTA writes clock64() at fixed points of its first 64 key tiles.
@@ -125,6 +136,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto bar_o_free = [&](int t) { return bar_x(7, t); };      // epilogue -> MMA: O_t has been read out
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
+#ifdef ROWMAX_TRACE
+    const long long trace_t0 = clock64();
+#endif
     if (tid == 256) ROWMAX_STAMP(2, 63, 0);
 
     const int n_pairs = (p.Sq + 2 * kTileM - 1) / (2 * kTileM);
@@ -171,7 +185,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     constexpr float p_off = static_cast<float>(PFormat<FP8, MODE>::kOffLog2);  // log2 of the P / row-sum scale
 
     if (wg == 3) {
-        reg_dec_48();
+        reg_dec<RegCfg<MODE>::kMma>();
         if (warp == 13 && lane == 0) {
             // ------------------------------------------------------------ TMA producer
             int kv_idx = 0;             // K/V tiles loaded so far (ring position), over all items
@@ -309,7 +323,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     } else if (wg == 2) {
         // ---------------------------------------------------------------- correction
-        reg_dec_80();
+        reg_dec<RegCfg<MODE>::kCorr>();
         const int r = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         int tiles[2] = {0, 0};
@@ -359,7 +373,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     } else {
         // ---------------------------------------------------------------- softmax + epilogue of query tile t
-        reg_inc_192();
+        reg_inc<RegCfg<MODE>::kSoftmax>();
         const int t = wg;
         const int r = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -390,6 +404,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_wait_ld();
                 if (r == 0) ROWMAX_STAMP(t, j, 1);
 
+                // Masked scores are set to -inf.  exact: their weight is then 0 by itself.  h15 family: a masked
+                // tile takes the clamped variant with the clamp one octave lower, at the input whose
+                // weight pattern is +0 (there a real score more than 126 octaves below its anchor also weighs 0,
+                // or a denormal, instead of 2^-126: nothing against a row sum >= 1).  pot and the partly emulated
+                // exact mode zero the masked weights explicitly (pot's floor 2^-20 is not nothing, and the
+                // polynomial route does not take -inf).  Keeping a masked variant out of the common modes
+                // makes their hot loop markedly faster.
                 const bool masked_tile = (j + 1) * kTileN > tile_limit;
                 const int col_limit = row_limit - j * kTileN;
                 if (masked_tile) {
@@ -423,8 +444,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 rs.c = make_float2(c_row, c_row);
                 rs.nmc = make_float2(nmc, nmc);
                 rs.two22 = p.two22;
+                rs.clamp_lo = 0.f;
+                if constexpr (kFam > 0) rs.clamp_lo = masked_tile ? h15_clamp_zero<kFam>() : h15_clamp_floor<kFam>();
                 float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                if (masked_tile) {
+                if ((MODE == kPot || MODE == kExactPoly) && masked_tile) {
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t pw[16];
@@ -433,13 +456,17 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         else tmem_st16(tS + cc * 16, pw);
                     }
                 } else {
-                    // h15: the clamp at -252 is a no-op unless some score of the warp's rows lies more than
-                    // 126 octaves below its running maximum; the row minimum (one more three-input pass)
-                    // tells, and the common case runs without the per-score clamp.
+                    // h15: the clamp is a no-op unless some score of the warp's rows lies more than 126 octaves
+                    // below its anchor; the row minimum (one more three-input pass) tells, and the common case
+                    // runs without the per-score clamp.  A tile with masked scores always takes the clamp.
                     bool clamp = false;
                     if constexpr (kFam > 0) {
-                        const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest scaled offset of the row
-                        clamp = __any_sync(0xffffffffu, !(lowest >= -125.0f * (1 << kFam)));
+                        if (masked_tile) {
+                            clamp = true;
+                        } else {
+                            const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest scaled offset of the row
+                            clamp = __any_sync(0xffffffffu, !(lowest >= -125.0f * (1 << kFam)));
+                        }
                     }
                     if (clamp) {
 #pragma unroll
@@ -471,7 +498,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
             // epilogue of this tile: O = v_descale * acc / l (the P offset cancels), LSE = ln2 * (m c + log2 l)
             if (q0 < p.Sq) {
-                const bool has_keys = l_run > 0.f;
+                const bool has_keys = (m_run != -INFINITY) && l_run > 0.f;
                 const float inv = has_keys ? p.v_descale / l_run : 0.f;
                 if (row < p.Sq && p.lse != nullptr) {
                     const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - p_off) : -INFINITY;
@@ -521,6 +548,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     tc_fence_before();
     __syncthreads();
     if (tid == 256) ROWMAX_STAMP(2, 63, 7);
+#ifdef ROWMAX_TRACE
+    if (tid == 0 && p.trace != nullptr && p.trace_block < 0) p.trace[blockIdx.x] = clock64() - trace_t0;   // per-CTA busy time
+#endif
     if (warp == 12) tmem_dealloc(tmem, kTmemCols);
 }
 

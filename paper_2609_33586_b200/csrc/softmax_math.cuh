@@ -141,6 +141,7 @@ struct RowScale {
     float2 c;      // multiplier of the raw score (c, or 2c for the doubled h15 input), both lanes
     float2 nmc;    // minus the scaled anchor (plus the P offset in exact mode), both lanes
     uint32_t two22;  // 1 << 22 held in a register (see imad)
+    float clamp_lo;  // h15 family, clamped variant: lower bound of the scaled offset (see w_h15_doubled_pair)
 };
 
 // Turns 32 consecutive scores of one row into weights.  Adds them (times 2^kOffLog2) into `acc`
@@ -173,7 +174,7 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
         } else if constexpr (h15_family_k(MODE) > 0) {
             // Eq. h15 on the input scaled by 2^K (K = 1: doubled): clamp, add 2^23 + 2^22 (rounds to the
             // integer n, ties to even), then (bits << (23 - K)) + bias builds the weight times 2^kOff.
-            w = w_h15_doubled_pair<kOff, CLAMP, h15_family_k(MODE)>(x, rs.two22);
+            w = w_h15_doubled_pair<kOff, CLAMP, h15_family_k(MODE)>(x, rs.two22, rs.clamp_lo);
         } else {
             // rs.c and rs.nmc carry the opposite sign in pot mode: x holds y = -(offset) >= 0
             w.x = pot_weight_from_y<kOff>(x.x);

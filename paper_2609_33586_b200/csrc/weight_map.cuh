@@ -52,14 +52,20 @@ __device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_fro
 // lane uses the shift-add (ALU pipe), the other the equivalent integer multiply-add (FMA pipe), which
 // balances the two pipes; `two22` must hold 1 << 22 and arrives in a register so that the
 // multiply-add is not turned back into a shift.  kOff scales the weight by 2^kOff (an exact exponent
-// shift) for the fp8 P formats.  kClamp = false skips the clamp at -126 * 2^K; the caller must know
-// that both inputs are at or above it.
+// shift) for the fp8 P formats.  kClamp = false skips the clamp; the caller must know that both
+// inputs are at or above -126 * 2^K.  The clamp value is -126 * 2^K (Eq. h15: the weight floor 2^-126);
+// the fused kernel passes -127 * 2^K in a key tile that holds masked scores: that input gives the
+// bit pattern of +0 (times 2^kOff), so a masked score (-inf) weighs exactly nothing.
+template <int K>
+__device__ __forceinline__ constexpr float h15_clamp_floor() { return -126.0f * (1 << K); }
+template <int K>
+__device__ __forceinline__ constexpr float h15_clamp_zero() { return -127.0f * (1 << K); }
 template <int kOff, bool kClamp = true, int K = 1>
-__device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22) {
+__device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22, float clamp_lo = h15_clamp_floor<K>()) {
     static_assert(K >= 1 && K <= 3, "family members k = 1, 2, 3");
     if constexpr (kClamp) {
-        x2.x = fmaxf(x2.x, -126.0f * (1 << K));
-        x2.y = fmaxf(x2.y, -126.0f * (1 << K));
+        x2.x = fmaxf(x2.x, clamp_lo);
+        x2.y = fmaxf(x2.y, clamp_lo);
     }
     float2 t;
     asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
