@@ -393,6 +393,19 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // first key index that some row of this tile cannot see (tile-uniform)
             const int tile_limit = p.causal ? min(p.Sk, q0 + shift + 1) : p.Sk;
             float m_run = -INFINITY, l_run = 0.f;
+            // h15 family at fp8: a lower bound of every raw score of this row that costs nothing per score.
+            // |q . k| <= (sum_i |q_i|) * max_i |k_i| and an e4m3 key element is at most 448 in magnitude, so
+            // s >= -448 * sum_i |q_i|.  When that bound already keeps the scaled offsets of a tile above the
+            // clamp, the tile needs neither the row-minimum pass nor the clamped variant.  The row of Q is
+            // read from shared memory (a sum does not care about the swizzle within the 128-byte row), which
+            // is safe while S_t(1) has not been issued, i.e. for items with at least two key tiles.
+            float score_floor = -INFINITY;
+            if constexpr (FP8 && kFam > 0 && D == 128) {
+                if (nt >= 2) {
+                    mbar_wait(bar_s_full(t), tiles & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);   // Q_t has landed
+                    score_floor = -448.0f * 1.02f * abs_sum_e4m3_row128(sQ + t * C::kTileBytes + r * 128);
+                }
+            }
             for (int j = 0; j < nt; ++j) {
                 mbar_wait(bar_s_full(t), (tiles + j) & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);
                 if (r == 0) ROWMAX_STAMP(t, j, 0);
@@ -463,7 +476,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     if constexpr (kFam > 0) {
                         if (masked_tile) {
                             clamp = true;
-                        } else {
+                        } else if (!__all_sync(0xffffffffu, (score_floor - m_use) * c_eff >= -125.0f * (1 << kFam))) {
                             const float lowest = (row_min128(s) - m_use) * c_eff;   // smallest scaled offset of the row
                             clamp = __any_sync(0xffffffffu, !(lowest >= -125.0f * (1 << kFam)));
                         }
