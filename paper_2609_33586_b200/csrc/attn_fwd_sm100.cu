@@ -39,16 +39,9 @@ struct WsCfg {
 
 // Register split of the 512 threads x 128 registers the CTA is launched with (setmaxnreg can only
 // redistribute that allocation; a larger total would make the increase wait for ever): softmax /
-// correction / MMA+TMA warpgroups.  The lattice modes (two weight variants in the loop, packed P words
-// kept alive) measured faster with more softmax registers, the exact modes with the other split.
-template <int MODE>
-struct RegCfg {
-    static constexpr bool kWide = !is_exact_like(MODE);
-    static constexpr int kSoftmax = kWide ? 208 : 192;
-    static constexpr int kCorr = kWide ? 56 : 80;
-    static constexpr int kMma = kWide ? 40 : 48;
-    static_assert(256 * kSoftmax + 128 * kCorr + 128 * kMma <= 512 * 128, "setmaxnreg targets exceed the launch allocation");
-};
+// correction / MMA+TMA warpgroups.
+constexpr int kRegSoftmax = 192, kRegCorr = 80, kRegMma = 48;
+static_assert(256 * kRegSoftmax + 128 * kRegCorr + 128 * kRegMma <= 512 * 128, "setmaxnreg targets exceed the launch allocation");
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
@@ -185,7 +178,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     constexpr float p_off = static_cast<float>(PFormat<FP8, MODE>::kOffLog2);  // log2 of the P / row-sum scale
 
     if (wg == 3) {
-        reg_dec<RegCfg<MODE>::kMma>();
+        reg_dec<kRegMma>();
         if (warp == 13 && lane == 0) {
             // ------------------------------------------------------------ TMA producer
             int kv_idx = 0;             // K/V tiles loaded so far (ring position), over all items
@@ -323,7 +316,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     } else if (wg == 2) {
         // ---------------------------------------------------------------- correction
-        reg_dec<RegCfg<MODE>::kCorr>();
+        reg_dec<kRegCorr>();
         const int r = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         int tiles[2] = {0, 0};
@@ -373,7 +366,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     } else {
         // ---------------------------------------------------------------- softmax + epilogue of query tile t
-        reg_inc<RegCfg<MODE>::kSoftmax>();
+        reg_inc<kRegSoftmax>();
         const int t = wg;
         const int r = tid & 127;
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
