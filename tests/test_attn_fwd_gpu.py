@@ -156,6 +156,21 @@ def test_huge_score_range_reaches_the_clamp(mode, dtype):
     assert st["ok"], st
 
 
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("scale_up", [1.0, 2.0])
+def test_h15_fp8_clamp_tests_agree(causal, scale_up):
+    # The fp8 h15 path skips its row-minimum pass when 448 * sum|q_i| already keeps every offset above
+    # the clamp.  scale_up = 1: the bound holds (Gaussian inputs); 2: scores four times larger, the bound
+    # fails and the row minimum decides (no clamp needed yet).  Both must match the oracle; items of one
+    # and of several key tiles are present (the bound is used only from two key tiles on).
+    wl = Workload("floor", 1, 2, 2, 640, 640, 128, causal, "fp8_e4m3", 46)
+    inp = make_inputs(wl)
+    inp.q_descale *= scale_up
+    inp.k_descale *= scale_up
+    st = compare(wl, orc.W_H15, inp, allow_output_rounding=scale_up > 1.0)
+    assert st["ok"], st
+
+
 @pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("tau", [8.0, 2.0])
 def test_deferred_rescale_matches_the_oracle_with_the_same_threshold(mode, tau):
