@@ -38,9 +38,9 @@ extern "C" {
 enum { ATTN_W_EXACT = 0, ATTN_W_POT = 1, ATTN_W_H15 = 2,
        ATTN_W_H15K2 = 3, ATTN_W_H15K3 = 4,     /* quarter- and eighth-octave members of the H15 family */
        ATTN_W_EXACT_POLY = 5 };               /* exact, a quarter of the 2^x evaluated by a cubic on the FMA pipe */
-enum { ATTN_IN_BF16 = 0, ATTN_IN_FP8_E4M3 = 1 };
+enum { ATTN_IN_BF16 = 0, ATTN_IN_FP8_E4M3 = 1, ATTN_IN_FP16 = 2 };
 /* format of the probability tile P fed to the P.V contraction, as reported by attn_get_schedule */
-enum { ATTN_P_BF16 = 0, ATTN_P_E4M3 = 1, ATTN_P_E5M2 = 2 };
+enum { ATTN_P_BF16 = 0, ATTN_P_E4M3 = 1, ATTN_P_E5M2 = 2, ATTN_P_FP16 = 3 };
 
 enum {
     ATTN_OK = 0,
@@ -58,17 +58,18 @@ enum {
 /*
  * attn_fwd — fused attention forward (Sec. 5.2; App. B.1 for the loop the weight map lives in).
  *
- *   q            (B, Sq, Hq, D)   bf16, or e4m3 bytes when in_dtype = ATTN_IN_FP8_E4M3; D contiguous
+ *   q            (B, Sq, Hq, D)   bf16, IEEE half (ATTN_IN_FP16; the FP16 rows of the timing tables in
+ *                                 App. B), or e4m3 bytes (ATTN_IN_FP8_E4M3); D contiguous
  *   k, v         (B, Sk, Hkv, D)  same storage type as q
  *   o            (B, Sq, Hq, D)   bf16, written
  *   lse          (B, Hq, Sq)      fp32, natural log, written; may be NULL
- *   D            64 or 128 for bf16; 128 for fp8
+ *   D            64 or 128 for bf16 and fp16; 128 for fp8
  *   causal       != 0: key j is visible to query i iff j <= i + Sk - Sq (aligned to the bottom-right
  *                corner); a row that sees no key gets O = 0 and LSE = -inf
  *   Hq, Hkv      query head h reads key/value head h / (Hq / Hkv)
  *   softmax_scale  multiplies q.k before the softmax (natural-exponent units)
  *   weight_mode  ATTN_W_EXACT / ATTN_W_POT / ATTN_W_H15 / ATTN_W_H15K2 / ATTN_W_H15K3 / ATTN_W_EXACT_POLY
- *   q/k/v_descale  per-tensor factors of the fp8 inputs (value = stored * descale); ignored for bf16
+ *   q/k/v_descale  per-tensor factors of the fp8 inputs (value = stored * descale); ignored for bf16 / fp16
  *
  * All tensors are contiguous; q, k, v, o must be 16-byte aligned.  In pot/h15 mode LSE is the log
  * of the approximated denominator.

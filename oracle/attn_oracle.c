@@ -37,7 +37,7 @@
 #endif
 
 enum { ORACLE_W_EXACT = 0, ORACLE_W_POT = 1, ORACLE_W_H15 = 2, ORACLE_W_H15K2 = 3, ORACLE_W_H15K3 = 4 };
-enum { ORACLE_IN_BF16 = 0, ORACLE_IN_FP8_E4M3 = 1 };
+enum { ORACLE_IN_BF16 = 0, ORACLE_IN_FP8_E4M3 = 1, ORACLE_IN_FP16 = 2 };
 enum { ORACLE_P_NONE = 0, ORACLE_P_BF16 = 1, ORACLE_P_E4M3 = 2, ORACLE_P_E5M2 = 3 };
 
 /* ---------------------------------------------------------------------------------------------
@@ -56,6 +56,22 @@ double oracle_decode_bf16(uint16_t h) {
         v = ldexp((double)f / 128.0, -126);
     } else {
         v = ldexp(1.0 + (double)f / 128.0, e - 127);
+    }
+    return sign ? -v : v;
+}
+
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+double oracle_decode_fp16(uint16_t h) {
+    int sign = (h >> 15) & 1;
+    int e = (h >> 10) & 0x1F;
+    int f = h & 0x3FF;
+    double v;
+    if (e == 0x1F) {
+        v = f ? NAN : INFINITY;
+    } else if (e == 0) {
+        v = ldexp((double)f / 1024.0, -14);
+    } else {
+        v = ldexp(1.0 + (double)f / 1024.0, e - 15);
     }
     return sign ? -v : v;
 }
@@ -181,6 +197,9 @@ static double* decode_tensor(const void* p, size_t n, int in_dtype) {
     if (in_dtype == ORACLE_IN_BF16) {
         const uint16_t* s = (const uint16_t*)p;
         for (size_t i = 0; i < n; ++i) out[i] = oracle_decode_bf16(s[i]);
+    } else if (in_dtype == ORACLE_IN_FP16) {
+        const uint16_t* s = (const uint16_t*)p;
+        for (size_t i = 0; i < n; ++i) out[i] = oracle_decode_fp16(s[i]);
     } else {
         const uint8_t* s = (const uint8_t*)p;
         for (size_t i = 0; i < n; ++i) out[i] = oracle_decode_e4m3(s[i]);
@@ -335,7 +354,7 @@ int oracle_attn(const void* q, const void* k, const void* v, int in_dtype, int B
                 int nthreads) {
     if (!q || !k || !v || !O || !LSE) return -1;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || D <= 0 || Hq % Hkv) return -2;
-    if (mode < 0 || mode > 4 || in_dtype < 0 || in_dtype > 1 || tile_n < 0) return -3;
+    if (mode < 0 || mode > 4 || in_dtype < 0 || in_dtype > 2 || tile_n < 0) return -3;
     if (tile_n == 0 && mode != ORACLE_W_EXACT) return -3;
     fesetround(FE_TONEAREST);
     if (!rows) nrows = Sq;
@@ -346,9 +365,9 @@ int oracle_attn(const void* q, const void* k, const void* v, int in_dtype, int B
         free(qd); free(kd); free(vd);
         return -4;
     }
-    double dq = in_dtype == ORACLE_IN_BF16 ? 1.0 : (double)q_descale;
-    double dk = in_dtype == ORACLE_IN_BF16 ? 1.0 : (double)k_descale;
-    double dv = in_dtype == ORACLE_IN_BF16 ? 1.0 : (double)v_descale;
+    double dq = in_dtype != ORACLE_IN_FP8_E4M3 ? 1.0 : (double)q_descale;
+    double dk = in_dtype != ORACLE_IN_FP8_E4M3 ? 1.0 : (double)k_descale;
+    double dv = in_dtype != ORACLE_IN_FP8_E4M3 ? 1.0 : (double)v_descale;
     double scale = (double)softmax_scale * dq * dk;
     float c32 = (float)(scale * 1.4426950408889634074); /* log2 e */
     int group = Hq / Hkv;

@@ -18,7 +18,7 @@ _SRC = _HERE / "attn_oracle.c"
 _LIB = _HERE / "liboracle.so"
 
 W_EXACT, W_POT, W_H15, W_H15K2, W_H15K3 = 0, 1, 2, 3, 4
-IN_BF16, IN_FP8_E4M3 = 0, 1
+IN_BF16, IN_FP8_E4M3, IN_FP16 = 0, 1, 2
 P_NONE, P_BF16, P_E4M3, P_E5M2 = 0, 1, 2, 3
 
 _lib = None
@@ -41,6 +41,8 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(str(build()))
         L.oracle_decode_bf16.restype = ctypes.c_double
         L.oracle_decode_bf16.argtypes = [ctypes.c_uint16]
+        L.oracle_decode_fp16.restype = ctypes.c_double
+        L.oracle_decode_fp16.argtypes = [ctypes.c_uint16]
         L.oracle_decode_e4m3.restype = ctypes.c_double
         L.oracle_decode_e4m3.argtypes = [ctypes.c_uint8]
         L.oracle_weight_map.restype = ctypes.c_int
@@ -57,6 +59,10 @@ def lib() -> ctypes.CDLL:
 
 def decode_bf16(bits: int) -> float:
     return lib().oracle_decode_bf16(int(bits))
+
+
+def decode_fp16(bits: int) -> float:
+    return lib().oracle_decode_fp16(int(bits))
 
 
 def decode_e4m3(bits: int) -> float:
@@ -80,12 +86,12 @@ def attn(q, k, v, *, in_dtype: int, causal: bool, softmax_scale: float, mode: in
          nthreads: int = 0):
     """Attention forward on raw storage arrays.
 
-    ``q`` is (B,Sq,Hq,D) and ``k``/``v`` are (B,Sk,Hkv,D): uint16 arrays holding bf16 bit patterns,
+    ``q`` is (B,Sq,Hq,D) and ``k``/``v`` are (B,Sk,Hkv,D): uint16 arrays holding bf16 (or, with IN_FP16, IEEE half) bit patterns,
     or uint8 arrays holding e4m3 bit patterns.  Returns a dict with ``O`` (B,Hq,R,D) and ``LSE``
     (B,Hq,R) in float64 over the R requested query rows, the tie bookkeeping arrays, and the
     number of threads the run used.
     """
-    want = np.uint16 if in_dtype == IN_BF16 else np.uint8
+    want = np.uint8 if in_dtype == IN_FP8_E4M3 else np.uint16
     q = np.ascontiguousarray(q)
     k = np.ascontiguousarray(k)
     v = np.ascontiguousarray(v)

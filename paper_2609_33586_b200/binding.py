@@ -12,8 +12,8 @@ from pathlib import Path
 import torch
 
 W_EXACT, W_POT, W_H15, W_H15K2, W_H15K3, W_EXACT_POLY = 0, 1, 2, 3, 4, 5
-IN_BF16, IN_FP8_E4M3 = 0, 1
-P_BF16, P_E4M3, P_E5M2 = 0, 1, 2
+IN_BF16, IN_FP8_E4M3, IN_FP16 = 0, 1, 2
+P_BF16, P_E4M3, P_E5M2, P_FP16 = 0, 1, 2, 3
 MODES = {"exact": W_EXACT, "pot": W_POT, "h15": W_H15, "h15k2": W_H15K2, "h15k3": W_H15K3,
          "exact_poly": W_EXACT_POLY}
 
@@ -105,6 +105,8 @@ def in_dtype_of(t: torch.Tensor) -> int:
         return IN_BF16
     if t.dtype == torch.float8_e4m3fn:
         return IN_FP8_E4M3
+    if t.dtype == torch.float16:
+        return IN_FP16
     raise TypeError(f"unsupported storage dtype {t.dtype}")
 
 
@@ -125,7 +127,7 @@ def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool,
              weight_mode: int, q_descale: float = 1.0, k_descale: float = 1.0, v_descale: float = 1.0,
              out: torch.Tensor | None = None, lse: torch.Tensor | None = None, return_lse: bool = True,
              rescale_tau: float | None = None, stream=None):
-    """q (B,Sq,Hq,D), k/v (B,Sk,Hkv,D): contiguous CUDA tensors, bf16 or float8_e4m3fn.
+    """q (B,Sq,Hq,D), k/v (B,Sk,Hkv,D): contiguous CUDA tensors, bf16, float16 or float8_e4m3fn.
     Returns (O bf16 (B,Sq,Hq,D), LSE fp32 (B,Hq,Sq) or None).  `rescale_tau` (bf16 inputs only) selects
     the deferred-rescale entry point attn_fwd_tau."""
     for t in (q, k, v):

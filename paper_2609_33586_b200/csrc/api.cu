@@ -10,7 +10,7 @@
 #include <cstdint>
 
 namespace rowmax {
-cudaError_t launch_attn_fwd(int D, bool fp8, int mode, const CUtensorMap& tq, const CUtensorMap& tk,
+cudaError_t launch_attn_fwd(int D, int in_type, int mode, const CUtensorMap& tq, const CUtensorMap& tk,
                             const CUtensorMap& tv, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cudaStream_t stream);
 cudaError_t status_word_address(int** out);
@@ -48,7 +48,7 @@ EncodeTiledFn encode_tiled_fn() {
 // Tensor (B, S, H, D) with D contiguous, viewed innermost-first as (D, H, S, B); one box is
 // 128 bytes along D by 128 rows along S of a single head, 128-byte swizzled in shared memory.
 // Rows past S read as zero.
-int make_tile_map(CUtensorMap* map, const void* base, bool fp8, int B, int S, int H, int D) {
+int make_tile_map(CUtensorMap* map, const void* base, bool fp8, bool half_in, int B, int S, int H, int D) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (enc == nullptr) return ATTN_ERR_CUDA;
     const cuuint64_t es = fp8 ? 1 : 2;
@@ -58,7 +58,8 @@ int make_tile_map(CUtensorMap* map, const void* base, bool fp8, int B, int S, in
                              static_cast<cuuint64_t>(S) * H * D * es};
     cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / es), 1, 128, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+    CUresult r = enc(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                              : (half_in ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), 4,
                      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -117,7 +118,7 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
                  float k_descale, float v_descale, float rescale_tau, void* stream) {
     if (!q || !k || !v || !o) return ATTN_ERR_NULLPTR;
     if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
-    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
+    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3 && in_dtype != ATTN_IN_FP16) return ATTN_ERR_BAD_ENUM;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return ATTN_ERR_BAD_SHAPE;
     if (D != 64 && D != 128) return ATTN_ERR_BAD_SHAPE;
     if (B > 65535 || Hq > 65535) return ATTN_ERR_BAD_SHAPE;  // grid y/z limits
@@ -131,6 +132,9 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
     if (fp8 && D != 128) return ATTN_ERR_UNSUPPORTED;
     if (!(rescale_tau >= 0.f) || !std::isfinite(rescale_tau) || rescale_tau > 32.f) return ATTN_ERR_BAD_VALUE;
     if (fp8 && rescale_tau != 0.f) return ATTN_ERR_UNSUPPORTED;   // the fp8 P formats have no headroom above the anchor
+    if (in_dtype == ATTN_IN_FP16 && rescale_tau != 0.f) return ATTN_ERR_UNSUPPORTED;   // fp16 P: not built
+    if (in_dtype == ATTN_IN_FP16 && weight_mode != ATTN_W_EXACT && weight_mode != ATTN_W_POT && weight_mode != ATTN_W_H15)
+        return ATTN_ERR_UNSUPPORTED;
     int rc = check_arch();
     if (rc != ATTN_OK) return rc;
 
@@ -154,11 +158,14 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
     if (rc != ATTN_OK) return rc;
 
     CUtensorMap tq, tk, tv;
-    if ((rc = make_tile_map(&tq, q, fp8, B, Sq, Hq, D)) != ATTN_OK) return rc;
-    if ((rc = make_tile_map(&tk, k, fp8, B, Sk, Hkv, D)) != ATTN_OK) return rc;
-    if ((rc = make_tile_map(&tv, v, fp8, B, Sk, Hkv, D)) != ATTN_OK) return rc;
+    const bool half_in = in_dtype == ATTN_IN_FP16;
+    if ((rc = make_tile_map(&tq, q, fp8, half_in, B, Sq, Hq, D)) != ATTN_OK) return rc;
+    if ((rc = make_tile_map(&tk, k, fp8, half_in, B, Sk, Hkv, D)) != ATTN_OK) return rc;
+    if ((rc = make_tile_map(&tv, v, fp8, half_in, B, Sk, Hkv, D)) != ATTN_OK) return rc;
 
-    cudaError_t e = rowmax::launch_attn_fwd(D, fp8, weight_mode, tq, tk, tv, p, static_cast<cudaStream_t>(stream));
+    static_assert(ATTN_IN_BF16 == rowmax::kInBF16 && ATTN_IN_FP8_E4M3 == rowmax::kInFP8 && ATTN_IN_FP16 == rowmax::kInFP16,
+                  "the kernel's storage-type codes are those of the C interface");
+    cudaError_t e = rowmax::launch_attn_fwd(D, in_dtype, weight_mode, tq, tk, tv, p, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(e);
         return e == cudaErrorInvalidValue ? ATTN_ERR_UNSUPPORTED : ATTN_ERR_CUDA;
@@ -191,7 +198,7 @@ int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* til
                       float* rescale_tau, int* pot_kmax, int* p_format, int* p_offset_log2) {
     (void)causal;
     if (D != 64 && D != 128) return ATTN_ERR_BAD_SHAPE;
-    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3) return ATTN_ERR_BAD_ENUM;
+    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3 && in_dtype != ATTN_IN_FP16) return ATTN_ERR_BAD_ENUM;
     if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
     const bool fp8 = in_dtype == ATTN_IN_FP8_E4M3;
     if (tile_m) *tile_m = rowmax::kTileM;
@@ -200,7 +207,7 @@ int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* til
     if (rescale_tau) *rescale_tau = 0.0f;
     if (pot_kmax) *pot_kmax = 20;
     const bool e4m3 = weight_mode == ATTN_W_EXACT || weight_mode == ATTN_W_EXACT_POLY || weight_mode == ATTN_W_H15K3;
-    if (p_format) *p_format = !fp8 ? ATTN_P_BF16 : (e4m3 ? ATTN_P_E4M3 : ATTN_P_E5M2);
+    if (p_format) *p_format = in_dtype == ATTN_IN_FP16 ? ATTN_P_FP16 : !fp8 ? ATTN_P_BF16 : (e4m3 ? ATTN_P_E4M3 : ATTN_P_E5M2);
     if (p_offset_log2) *p_offset_log2 = !fp8 ? 0 : (e4m3 ? 8 : 15);
     return ATTN_OK;
 }

@@ -98,10 +98,14 @@ __device__ __forceinline__ WorkItem decode_item(int w, const AttnParams& p, int 
 
 }  // namespace
 
-template <int D, bool FP8, int MODE>
+// IN: storage type of q, k, v (kInBF16 / kInFP8 / kInFP16).  P has the type of V at 16 bits (the f16
+// kind wants both MMA operands in one format) and one of the two fp8 formats at 8 bits.
+template <int D, int IN, int MODE>
 __global__ void __launch_bounds__(512, 1)
 attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+    constexpr bool FP8 = IN == kInFP8;
+    constexpr bool HALF = IN == kInFP16;
     using C = TileCfg<D, FP8>;
     using W = WsCfg<D, FP8>;
     constexpr int NS = W::kSlots;
@@ -171,8 +175,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto tmem_S = [&](int t) { return tmem + 128u * t; };
     auto tmem_O = [&](int t) { return tmem + 256u + 128u * t; };
 
-    constexpr uint32_t fmt_ab = FP8 ? kFmtE4M3 : kFmtBF16;
-    constexpr uint32_t fmt_p = FP8 ? (PFormat<FP8, MODE>::kE4M3 ? kFmtE4M3 : kFmtE5M2) : kFmtBF16;
+    constexpr uint32_t fmt_16 = HALF ? kFmtF16 : kFmtBF16;
+    constexpr uint32_t fmt_ab = FP8 ? kFmtE4M3 : fmt_16;
+    constexpr uint32_t fmt_p = FP8 ? (PFormat<FP8, MODE>::kE4M3 ? kFmtE4M3 : kFmtE5M2) : fmt_16;
     constexpr uint32_t idesc_s = umma_idesc(fmt_ab, fmt_ab, false, false, kTileM, kTileN);
     constexpr uint32_t idesc_pv = umma_idesc(fmt_p, fmt_ab, false, true, kTileM, D);
     constexpr float p_off = static_cast<float>(PFormat<FP8, MODE>::kOffLog2);  // log2 of the P / row-sum scale
@@ -457,7 +462,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t pw[16];
-                        weights_chunk32<FP8, MODE, true>(s[cc], rs, col_limit - cc * 32, acc, pw);
+                        weights_chunk32<FP8, MODE, true, true, HALF>(s[cc], rs, col_limit - cc * 32, acc, pw);
                         if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                         else tmem_st16(tS + cc * 16, pw);
                     }
@@ -478,7 +483,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) {
                             uint32_t pw[16];
-                            weights_chunk32<FP8, MODE, false, true>(s[cc], rs, 32, acc, pw);
+                            weights_chunk32<FP8, MODE, false, true, HALF>(s[cc], rs, 32, acc, pw);
                             if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                             else tmem_st16(tS + cc * 16, pw);
                         }
@@ -486,7 +491,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) {
                             uint32_t pw[16];
-                            weights_chunk32<FP8, MODE, false, false>(s[cc], rs, 32, acc, pw);
+                            weights_chunk32<FP8, MODE, false, false, HALF>(s[cc], rs, 32, acc, pw);
                             if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                             else tmem_st16(tS + cc * 16, pw);
                         }
@@ -563,11 +568,11 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 // ------------------------------------------------------------------------------------------------
 // Host launcher
 // ------------------------------------------------------------------------------------------------
-template <int D, bool FP8, int MODE>
+template <int D, int IN, int MODE>
 static cudaError_t launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              const AttnParams& p, cudaStream_t stream) {
-    using W = WsCfg<D, FP8>;
-    auto kern = attn_fwd_ws_kernel<D, FP8, MODE>;
+    using W = WsCfg<D, IN == kInFP8>;
+    auto kern = attn_fwd_ws_kernel<D, IN, MODE>;
     // per-device launch set-up: the shared-memory opt-in of this instance and the SM count
     static bool configured[64] = {};
     static int sm_counts[64] = {};
@@ -591,25 +596,34 @@ static cudaError_t launch_ws(const CUtensorMap& tq, const CUtensorMap& tk, const
     return cudaGetLastError();
 }
 
-template <int D, bool FP8>
+template <int D, int IN>
 static cudaError_t dispatch_mode(int mode, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                  const AttnParams& p, cudaStream_t stream) {
     switch (mode) {
-        case kExact: return launch_ws<D, FP8, kExact>(tq, tk, tv, p, stream);
-        case kPot: return launch_ws<D, FP8, kPot>(tq, tk, tv, p, stream);
-        case kH15K2: return launch_ws<D, FP8, kH15K2>(tq, tk, tv, p, stream);
-        case kH15K3: return launch_ws<D, FP8, kH15K3>(tq, tk, tv, p, stream);
-        case kExactPoly: return launch_ws<D, FP8, kExactPoly>(tq, tk, tv, p, stream);
-        default: return launch_ws<D, FP8, kH15>(tq, tk, tv, p, stream);
+        case kExact: return launch_ws<D, IN, kExact>(tq, tk, tv, p, stream);
+        case kPot: return launch_ws<D, IN, kPot>(tq, tk, tv, p, stream);
+        case kH15: return launch_ws<D, IN, kH15>(tq, tk, tv, p, stream);
+        default: break;
     }
+    if constexpr (IN != kInFP16) {   // the family members and the emulated control are built for bf16 and fp8 only
+        switch (mode) {
+            case kH15K2: return launch_ws<D, IN, kH15K2>(tq, tk, tv, p, stream);
+            case kH15K3: return launch_ws<D, IN, kH15K3>(tq, tk, tv, p, stream);
+            case kExactPoly: return launch_ws<D, IN, kExactPoly>(tq, tk, tv, p, stream);
+            default: break;
+        }
+    }
+    return cudaErrorInvalidValue;
 }
 
 // Returns cudaErrorInvalidValue for a combination that is not built.
-cudaError_t launch_attn_fwd(int D, bool fp8, int mode, const CUtensorMap& tq, const CUtensorMap& tk,
+cudaError_t launch_attn_fwd(int D, int in_type, int mode, const CUtensorMap& tq, const CUtensorMap& tk,
                             const CUtensorMap& tv, const AttnParams& p, cudaStream_t stream) {
-    if (!fp8 && D == 128) return dispatch_mode<128, false>(mode, tq, tk, tv, p, stream);
-    if (!fp8 && D == 64) return dispatch_mode<64, false>(mode, tq, tk, tv, p, stream);
-    if (fp8 && D == 128) return dispatch_mode<128, true>(mode, tq, tk, tv, p, stream);
+    if (in_type == kInBF16 && D == 128) return dispatch_mode<128, kInBF16>(mode, tq, tk, tv, p, stream);
+    if (in_type == kInBF16 && D == 64) return dispatch_mode<64, kInBF16>(mode, tq, tk, tv, p, stream);
+    if (in_type == kInFP16 && D == 128) return dispatch_mode<128, kInFP16>(mode, tq, tk, tv, p, stream);
+    if (in_type == kInFP16 && D == 64) return dispatch_mode<64, kInFP16>(mode, tq, tk, tv, p, stream);
+    if (in_type == kInFP8 && D == 128) return dispatch_mode<128, kInFP8>(mode, tq, tk, tv, p, stream);
     return cudaErrorInvalidValue;
 }
 

@@ -8,6 +8,8 @@ namespace rowmax {
 constexpr int kTileM = 128;  // query rows per tile
 constexpr int kTileN = 128;  // keys per tile
 
+// storage type of q, k, v (the values of ATTN_IN_* in the C interface)
+enum InType : int { kInBF16 = 0, kInFP8 = 1, kInFP16 = 2 };
 enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4, kExactPoly = 5 };
 // modes whose weight is 2^x itself (with the P offset folded into x)
 __host__ __device__ constexpr bool is_exact_like(int mode) { return mode == kExact || mode == kExactPoly; }

@@ -182,6 +182,7 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr, uint32_t lbo
 // Instruction descriptor (32 bit) for kind::f16 / kind::f8f6f4, fp32 accumulate:
 // [4,6) D format (1 = f32), [7,10) A format, [10,13) B format, bit 15 A MN-major, bit 16 B MN-major,
 // [17,23) N >> 3, [24,29) M >> 4.
+constexpr uint32_t kFmtF16 = 0;   // kind::f16
 constexpr uint32_t kFmtBF16 = 1;  // kind::f16
 constexpr uint32_t kFmtE4M3 = 0;  // kind::f8f6f4
 constexpr uint32_t kFmtE5M2 = 1;  // kind::f8f6f4

@@ -176,10 +176,10 @@ struct RowScale {
 
 // Turns 32 consecutive scores of one row into weights.  Adds them (times 2^kOffLog2) into `acc`
 // (two independent packed accumulators, summed by the caller)
-// and writes the packed P words: 16 words of 2 bf16, or 8 words of 4 fp8.  In a MASKED tile
+// and writes the packed P words: 16 words of 2 bf16 (2 fp16 with HALFP), or 8 words of 4 fp8.  In a MASKED tile
 // columns >= limit are masked: their scores already hold -inf and their weights are forced to 0.
 // CLAMP = false (h15 only) may be used when every doubled offset of the chunk is known to be >= -252.
-template <bool FP8, int MODE, bool MASKED, bool CLAMP = true>
+template <bool FP8, int MODE, bool MASKED, bool CLAMP = true, bool HALFP = false>
 __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const RowScale& rs, int limit,
                                                 float2 (&acc)[2], uint32_t* pw) {
     constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
@@ -215,7 +215,9 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             if (2 * i + 1 >= limit) w.y = 0.f;
         }
         acc[i & 1] = fadd2(acc[i & 1], w);
-        if constexpr (!FP8) {
+        if constexpr (!FP8 && HALFP) {
+            pw[i] = pack_f16x2_rn(w.x, w.y);   // fp16 P: exact for the lattice weights down to 2^-14, rounded to nearest otherwise
+        } else if constexpr (!FP8) {
             if constexpr (is_exact_like(MODE)) pw[i] = pack_bf16_rn(w.x, w.y);
             else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: at most 3 fraction bits
         } else {

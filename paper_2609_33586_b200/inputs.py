@@ -31,7 +31,7 @@ class Workload:
     Sk: int
     D: int
     causal: bool
-    in_dtype: str            # "bf16" | "fp8_e4m3"
+    in_dtype: str            # "bf16" | "fp16" | "fp8_e4m3"
     seed: int
     peaked_keys: bool = False  # multiply every key row by its own U(0.5, 2) factor
 
@@ -73,6 +73,8 @@ class Inputs:
 def _to_storage(x: torch.Tensor, in_dtype: str):
     if in_dtype == "bf16":
         return x.to(torch.bfloat16), 1.0
+    if in_dtype == "fp16":
+        return x.to(torch.float16), 1.0
     if in_dtype == "fp8_e4m3":
         descale = float(np.float32(float(x.abs().max()) / E4M3_MAX))  # the fp32 value the C interface receives
         y = (x / descale).clamp(-E4M3_MAX, E4M3_MAX).to(torch.float8_e4m3fn)
@@ -97,9 +99,9 @@ def make_inputs(w: Workload) -> Inputs:
 
 
 def storage_bits(t: torch.Tensor) -> np.ndarray:
-    """Raw bit patterns of a bf16 (-> uint16) or e4m3 (-> uint8) CPU tensor."""
+    """Raw bit patterns of a bf16 or fp16 (-> uint16) or e4m3 (-> uint8) CPU tensor."""
     t = t.contiguous().cpu()
-    if t.dtype == torch.bfloat16:
+    if t.dtype == torch.bfloat16 or t.dtype == torch.float16:
         return t.view(torch.int16).numpy().view(np.uint16)
     if t.dtype == torch.float8_e4m3fn:
         return t.view(torch.uint8).numpy()

@@ -18,6 +18,7 @@ from paper_2609_33586_b200.inputs import Inputs, Workload, make_inputs, storage_
 
 TIE_EPS = 2.0 ** -16
 TOL = {"bf16": {"o_max": 1e-2, "o_mean": 1e-3, "lse": 1e-3},
+       "fp16": {"o_max": 1e-2, "o_mean": 1e-3, "lse": 1e-3},
        "fp8_e4m3": {"o_max": 5e-2, "o_mean": None, "lse": 1e-3}}
 # Exact mode on fp8 inputs stores P in e4m3 (3 fraction bits, as the paper's baseline kernel does).  On
 # causal rows that see fewer than 16 keys two or three comparable weights carry the whole row, their
@@ -37,7 +38,7 @@ def run_cuda(wl: Workload, inp: Inputs, mode: int, device="cuda:0", tau=None):
 
 
 def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None, model_p_storage=False):
-    dt = orc.IN_BF16 if wl.in_dtype == "bf16" else orc.IN_FP8_E4M3
+    dt = {"bf16": orc.IN_BF16, "fp16": orc.IN_FP16, "fp8_e4m3": orc.IN_FP8_E4M3}[wl.in_dtype]
     sch = binding.get_schedule(wl.D, dt, mode, wl.causal)
     if mode == binding.W_EXACT_POLY:
         mode = orc.W_EXACT      # the partly emulated exponential is held to the exact definition

@@ -156,6 +156,38 @@ def test_huge_score_range_reaches_the_clamp(mode, dtype):
     assert st["ok"], st
 
 
+FP16_SHAPES = [
+    Workload("fp16_small", 2, 4, 2, 320, 448, 128, True, "fp16", 51),
+    Workload("fp16_d64", 1, 2, 2, 384, 384, 64, False, "fp16", 52),
+    Workload("fp16_peaked", 1, 4, 4, 512, 512, 128, True, "fp16", 53, peaked_keys=True),
+]
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("wl", FP16_SHAPES, ids=lambda w: w.name)
+def test_fp16_inputs_small_shapes(wl, mode):
+    # IEEE half inputs (the FP16 rows of the timing tables in App. B); same tolerances as bf16
+    st = compare(wl, mode)
+    assert st["ok"], st
+
+
+def test_fp16_inputs_reject_what_is_not_built():
+    q = torch.zeros(1, 128, 2, 128, dtype=torch.float16, device="cuda")
+    args = (q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128, 128, 1, 0.1)
+    assert binding.attn_fwd_raw(*args, binding.W_H15K2, binding.IN_FP16, 1.0, 1.0, 1.0, None) == -8
+    assert binding.attn_fwd_raw(*args, binding.W_EXACT_POLY, binding.IN_FP16, 1.0, 1.0, 1.0, None) == -8
+    assert binding.attn_fwd_raw(*args, binding.W_H15, binding.IN_FP16, 1.0, 1.0, 1.0, None, rescale_tau=4.0) == -8
+    assert binding.get_schedule(128, binding.IN_FP16, binding.W_H15, True)["p_format"] == binding.P_FP16
+
+
+@pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_H15])
+def test_fp16_inputs_full_size_8k_on_sampled_rows(mode):
+    wl = Workload("causal_8k_fp16", 1, 16, 16, 8192, 8192, 128, True, "fp16", 54)
+    rows = np.unique(np.concatenate([np.arange(0, 8192, 509), [127, 128, 255, 256, 8191]])).astype(np.int32)
+    st = compare(wl, mode, rows=rows)
+    assert st["ok"], st
+
+
 @pytest.mark.parametrize("causal", [True, False])
 @pytest.mark.parametrize("scale_up", [1.0, 2.0])
 def test_h15_fp8_clamp_tests_agree(causal, scale_up):

@@ -201,6 +201,16 @@ def test_bf16_decoder_matches_torch_for_every_pattern():
     assert np.array_equal(np.signbit(ref[~both_nan]), np.signbit(got[~both_nan]))
 
 
+def test_fp16_decoder_matches_torch_for_every_pattern():
+    bits = np.arange(65536, dtype=np.uint16)
+    ref = torch.from_numpy(bits.view(np.int16)).view(torch.float16).to(torch.float64).numpy()
+    got = np.array([orc.decode_fp16(int(b)) for b in bits])
+    both_nan = np.isnan(ref) & np.isnan(got)
+    assert np.all((ref == got) | both_nan)
+    assert np.array_equal(np.signbit(ref[~both_nan]), np.signbit(got[~both_nan]))
+    assert got[0x7BFF] == 65504.0 and got[0x0001] == 2.0 ** -24
+
+
 def test_e4m3_decoder_matches_torch_for_every_pattern():
     bits = np.arange(256, dtype=np.uint8)
     ref = torch.from_numpy(bits).view(torch.float8_e4m3fn).to(torch.float64).numpy()
