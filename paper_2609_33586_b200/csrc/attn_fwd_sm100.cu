@@ -396,10 +396,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // s >= -448 * sum_i |q_i|.  When that bound already keeps the scaled offsets of a tile above the
             // clamp, the tile needs neither the row-minimum pass nor the clamped variant.  The row of Q is
             // read from shared memory (a sum does not care about the swizzle within the 128-byte row), which
-            // is safe while S_t(1) has not been issued, i.e. for items with at least two key tiles.
+            // is safe while S_t(1) has not been issued, i.e. for items with at least two key tiles (used from four on).
             float score_floor = -INFINITY;
             if constexpr (FP8 && kFam > 0 && D == 128) {
-                if (nt >= 2) {
+                if (nt >= 4) {   // the sum costs about three row-minimum passes
                     mbar_wait(bar_s_full(t), tiles & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);   // Q_t has landed
                     score_floor = -448.0f * 1.02f * abs_sum_e4m3_row128(sQ + t * C::kTileBytes + r * 128);
                 }
