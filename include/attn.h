@@ -63,7 +63,7 @@ enum {
  *   k, v         (B, Sk, Hkv, D)  same storage type as q
  *   o            (B, Sq, Hq, D)   bf16, written
  *   lse          (B, Hq, Sq)      fp32, natural log, written; may be NULL
- *   D            64 or 128 for bf16 and fp16; 128 for fp8
+ *   D            64 or 128
  *   causal       != 0: key j is visible to query i iff j <= i + Sk - Sq (aligned to the bottom-right
  *                corner); a row that sees no key gets O = 0 and LSE = -inf
  *   Hq, Hkv      query head h reads key/value head h / (Hq / Hkv)

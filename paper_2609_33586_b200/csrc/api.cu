@@ -46,7 +46,8 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // Tensor (B, S, H, D) with D contiguous, viewed innermost-first as (D, H, S, B); one box is
-// 128 bytes along D by 128 rows along S of a single head, 128-byte swizzled in shared memory.
+// 128 bytes along D (64 when a row has only 64: fp8 with D = 64) by 128 rows along S of a single
+// head, swizzled in shared memory with that span.
 // Rows past S read as zero.
 int make_tile_map(CUtensorMap* map, const void* base, bool fp8, bool half_in, int B, int S, int H, int D) {
     EncodeTiledFn enc = encode_tiled_fn();
@@ -56,12 +57,14 @@ int make_tile_map(CUtensorMap* map, const void* base, bool fp8, bool half_in, in
                           static_cast<cuuint64_t>(B)};
     cuuint64_t strides[3] = {static_cast<cuuint64_t>(D) * es, static_cast<cuuint64_t>(H) * D * es,
                              static_cast<cuuint64_t>(S) * H * D * es};
-    cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / es), 1, 128, 1};
+    const cuuint64_t row_bytes = static_cast<cuuint64_t>(D) * es;
+    const cuuint64_t span = row_bytes >= 128 ? 128 : 64;   // swizzle span: a whole row when it has only 64 bytes
+    cuuint32_t box[4] = {static_cast<cuuint32_t>(span / es), 1, 128, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                               : (half_in ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), 4,
                      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     span == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         g_last_cuda_error = static_cast<int>(r);
@@ -129,7 +132,6 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
                 !std::isfinite(k_descale) || !std::isfinite(v_descale)))
         return ATTN_ERR_BAD_VALUE;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return ATTN_ERR_MISALIGNED;
-    if (fp8 && D != 128) return ATTN_ERR_UNSUPPORTED;
     if (!(rescale_tau >= 0.f) || !std::isfinite(rescale_tau) || rescale_tau > 32.f) return ATTN_ERR_BAD_VALUE;
     if (fp8 && rescale_tau != 0.f) return ATTN_ERR_UNSUPPORTED;   // the fp8 P formats have no headroom above the anchor
     if (in_dtype == ATTN_IN_FP16 && rescale_tau != 0.f) return ATTN_ERR_UNSUPPORTED;   // fp16 P: not built

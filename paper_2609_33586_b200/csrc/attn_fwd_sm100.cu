@@ -225,7 +225,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // The whole warp walks the loop (so addresses and descriptors stay warp-uniform values);
             // one elected lane issues the MMAs and commits.
             const bool leader = elect_one();
-            constexpr uint32_t desc_hi = umma_desc_hi_sw128(1024);
+            constexpr uint32_t desc_hi = umma_desc_hi_sw(C::kSwizzle);
             const uint32_t q_lo0 = umma_desc_lo(sQ, 16);
             const uint32_t ring_lo_k = umma_desc_lo(sRing, 16);               // K tiles: K-major
             const uint32_t ring_lo_v = umma_desc_lo(sRing, C::kBoxBytes);     // V tiles: MN-major, LBO = next 128-byte column block
@@ -234,14 +234,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const uint32_t q_lo = q_lo0 + t * kTileLo;
 #pragma unroll
                 for (int ks = 0; ks < C::kQkSteps; ++ks) {
-                    const uint32_t off = ((ks / 4) * C::kBoxBytes + (ks % 4) * 32) >> 4;
+                    const uint32_t off = ((ks / C::kStepsPerBox) * C::kBoxBytes + (ks % C::kStepsPerBox) * 32) >> 4;
                     umma_ss_lo<FP8>(tmem_S(t), q_lo + off, k_lo + off, desc_hi, idesc_s, ks > 0 ? 1u : 0u);
                 }
             };
             auto issue_pv = [&](int t, uint32_t v_lo, bool accumulate) {
 #pragma unroll
                 for (int ks = 0; ks < C::kPvSteps; ++ks) {
-                    const uint32_t off = (ks * C::kUmmaK * 128) >> 4;
+                    const uint32_t off = (ks * C::kUmmaK * C::kSwizzle) >> 4;   // kUmmaK keys down the MN-major V tile
                     umma_ts_lo<FP8>(tmem_O(t), tmem_S(t) + ks * 8, v_lo + off, desc_hi, idesc_pv,
                                     (accumulate || ks > 0) ? 1u : 0u);
                 }
@@ -395,13 +395,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // |q . k| <= (sum_i |q_i|) * max_i |k_i| and an e4m3 key element is at most 448 in magnitude, so
             // s >= -448 * sum_i |q_i|.  When that bound already keeps the scaled offsets of a tile above the
             // clamp, the tile needs neither the row-minimum pass nor the clamped variant.  The row of Q is
-            // read from shared memory (a sum does not care about the swizzle within the 128-byte row), which
+            // read from shared memory (a sum does not care about the swizzle, which stays within the row), which
             // is safe while S_t(1) has not been issued, i.e. for items with at least two key tiles (used from four on).
             float score_floor = -INFINITY;
-            if constexpr (FP8 && kFam > 0 && D == 128) {
+            if constexpr (FP8 && kFam > 0) {
                 if (nt >= 4) {   // the sum costs about three row-minimum passes
                     mbar_wait(bar_s_full(t), tiles & 1, wctx, (kRoleSoftmax << 8) | kBarSFull);   // Q_t has landed
-                    score_floor = -448.0f * 1.02f * abs_sum_e4m3_row128(sQ + t * C::kTileBytes + r * 128);
+                    score_floor = -448.0f * 1.02f * abs_sum_e4m3_row<D / 16>(sQ + t * C::kTileBytes + r * D);
                 }
             }
             for (int j = 0; j < nt; ++j) {
@@ -624,6 +624,7 @@ cudaError_t launch_attn_fwd(int D, int in_type, int mode, const CUtensorMap& tq,
     if (in_type == kInFP16 && D == 128) return dispatch_mode<128, kInFP16>(mode, tq, tk, tv, p, stream);
     if (in_type == kInFP16 && D == 64) return dispatch_mode<64, kInFP16>(mode, tq, tk, tv, p, stream);
     if (in_type == kInFP8 && D == 128) return dispatch_mode<128, kInFP8>(mode, tq, tk, tv, p, stream);
+    if (in_type == kInFP8 && D == 64) return dispatch_mode<64, kInFP8>(mode, tq, tk, tv, p, stream);
     return cudaErrorInvalidValue;
 }
 

@@ -232,6 +232,11 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
 __host__ __device__ constexpr uint32_t umma_desc_hi_sw128(uint32_t sbo_bytes) {
     return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
 }
+// Same for a swizzle span of 128 or 64 bytes (layout type 2 or 4); the stride between groups of
+// eight rows is eight swizzle rows.
+__host__ __device__ constexpr uint32_t umma_desc_hi_sw(uint32_t swizzle_bytes) {
+    return (((8u * swizzle_bytes) >> 4) & 0x3FFFu) | (1u << 14) | ((swizzle_bytes == 128u ? 2u : 4u) << 29);
+}
 __device__ __forceinline__ uint32_t umma_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
     return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }

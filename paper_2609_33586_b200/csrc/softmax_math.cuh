@@ -18,14 +18,17 @@ template <int D, bool FP8>
 struct TileCfg {
     static constexpr int kElem = FP8 ? 1 : 2;
     static constexpr int kRowBytes = D * kElem;
-    static constexpr int kBoxElems = 128 / kElem;           // one 128-byte swizzle row
-    static constexpr int kBoxes = kRowBytes / 128;          // boxes per tile along D
-    static constexpr int kBoxBytes = 128 * 128;             // 128 rows x 128 bytes
+    // Swizzle span of the shared-memory tiles: 128 bytes, or 64 when a row has only 64 (fp8, D = 64).
+    static constexpr int kSwizzle = kRowBytes >= 128 ? 128 : 64;
+    static constexpr int kBoxElems = kSwizzle / kElem;      // one swizzle row
+    static constexpr int kBoxes = kRowBytes / kSwizzle;     // boxes per tile along D
+    static constexpr int kBoxBytes = 128 * kSwizzle;        // 128 rows x one swizzle row
     static constexpr int kTileBytes = kBoxes * kBoxBytes;   // 128 rows x D
+    static constexpr int kStepsPerBox = kSwizzle / 32;      // MMA steps (32 bytes along K) per swizzle row
     static constexpr int kUmmaK = 32 / kElem;               // elements per MMA along K (32 bytes)
     static constexpr int kQkSteps = D / kUmmaK;
     static constexpr int kPvSteps = kTileN / kUmmaK;
-    static_assert(kRowBytes % 128 == 0, "row must be a whole number of 128-byte swizzle rows");
+    static_assert(kRowBytes % kSwizzle == 0, "row must be a whole number of swizzle rows");
 };
 
 // P is stored as weight * 2^kPOff so that it fills the range of its fp8 format: e4m3 holds the
@@ -137,13 +140,14 @@ __device__ __forceinline__ float row_min128(const uint32_t (&s)[4][32]) {
     return fminf(min3(m[0], m[1], m[2]), min3(m[3], m[4], min3(m[5], m[6], m[7])));
 }
 
-// Sum of |x| over the 128 e4m3 bytes at a 128-byte aligned shared-memory address, rounded up a little
+// Sum of |x| over the 16 * CHUNKS e4m3 bytes (128 or 64) at a 16-byte aligned shared-memory address, rounded up a little
 // (the caller adds its own margin): pairs are widened to fp16 (exact), summed in eight fp16 lanes of at
 // most 16 terms each (each partial sum <= 7168, so no overflow and an error below 0.5 %), then in fp32.
-__device__ __forceinline__ float abs_sum_e4m3_row128(uint32_t saddr) {
+template <int CHUNKS>
+__device__ __forceinline__ float abs_sum_e4m3_row(uint32_t saddr) {
     uint32_t acc[4] = {0u, 0u, 0u, 0u};   // four f16x2 accumulators
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < CHUNKS; ++c) {
         uint32_t w[4];
         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(saddr + 16u * c));
 #pragma unroll

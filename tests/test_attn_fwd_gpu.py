@@ -171,6 +171,29 @@ def test_fp16_inputs_small_shapes(wl, mode):
     assert st["ok"], st
 
 
+FP8_D64_SHAPES = [
+    Workload("fp8_d64_small", 2, 4, 2, 320, 448, 64, True, "fp8_e4m3", 56),
+    Workload("fp8_d64_noncausal", 1, 2, 2, 384, 384, 64, False, "fp8_e4m3", 57),
+    Workload("fp8_d64_ragged", 1, 3, 1, 200, 333, 64, True, "fp8_e4m3", 58, peaked_keys=True),
+]
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("wl", FP8_D64_SHAPES, ids=lambda w: w.name)
+def test_fp8_head_dim_64_small_shapes(wl, mode):
+    # 64-byte rows: the shared-memory tiles use the 64-byte swizzle
+    st = compare(wl, mode, model_p_storage=True)
+    assert st["ok"], st
+
+
+@pytest.mark.parametrize("mode", [orc.W_EXACT, orc.W_H15])
+def test_fp8_head_dim_64_causal_4k_on_sampled_rows(mode):
+    wl = Workload("causal_4k_fp8_d64", 1, 16, 16, 4096, 4096, 64, True, "fp8_e4m3", 59)
+    rows = np.unique(np.concatenate([np.arange(0, 4096, 251), [127, 128, 255, 256, 4095]])).astype(np.int32)
+    st = compare(wl, mode, rows=rows)
+    assert st["ok"], st
+
+
 def test_fp16_inputs_reject_what_is_not_built():
     q = torch.zeros(1, 128, 2, 128, dtype=torch.float16, device="cuda")
     args = (q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128, 128, 1, 0.1)
