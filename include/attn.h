@@ -51,7 +51,7 @@ enum {
     ATTN_ERR_UNSUPPORTED_ARCH = -5, /* current device is not compute capability 10.x */
     ATTN_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed; see attn_last_cuda_error */
     ATTN_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired; see attn_device_status */
-    ATTN_ERR_UNSUPPORTED = -8,      /* valid arguments, combination not built (e.g. fp8 with D = 64) */
+    ATTN_ERR_UNSUPPORTED = -8,      /* valid arguments, combination not built (e.g. a deferred rescale on fp8 inputs) */
     ATTN_ERR_BAD_VALUE = -9         /* softmax_scale or an fp8 descale is not positive and finite */
 };
 
@@ -69,6 +69,7 @@ enum {
  *   Hq, Hkv      query head h reads key/value head h / (Hq / Hkv)
  *   softmax_scale  multiplies q.k before the softmax (natural-exponent units)
  *   weight_mode  ATTN_W_EXACT / ATTN_W_POT / ATTN_W_H15 / ATTN_W_H15K2 / ATTN_W_H15K3 / ATTN_W_EXACT_POLY
+ *                (fp16 inputs: the first three; the others return ATTN_ERR_UNSUPPORTED)
  *   q/k/v_descale  per-tensor factors of the fp8 inputs (value = stored * descale); ignored for bf16 / fp16
  *
  * All tensors are contiguous; q, k, v, o must be 16-byte aligned.  In pot/h15 mode LSE is the log
@@ -85,8 +86,8 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
  * row's anchor only when it exceeds the anchor by more than rescale_tau octaves of the scaled score,
  * so O is rescaled far less often and x can be positive (Eq. h15 covers both signs).  Exact mode is
  * unchanged by this up to rounding; pot and h15 results differ from rescale_tau = 0 because the
- * lattice is anchored at the lagging maximum.  bf16 inputs only (ATTN_ERR_UNSUPPORTED for fp8: its P
- * formats have no headroom above the anchor); 0 <= rescale_tau <= 32, else ATTN_ERR_BAD_VALUE.
+ * lattice is anchored at the lagging maximum.  bf16 inputs only (ATTN_ERR_UNSUPPORTED for fp8, whose P
+ * formats have no headroom above the anchor, and for fp16); 0 <= rescale_tau <= 32, else ATTN_ERR_BAD_VALUE.
  * attn_fwd is attn_fwd_tau with rescale_tau = 0.
  */
 int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* lse,
@@ -97,7 +98,8 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
 /*
  * attn_weight_map — applies the weight map of `weight_mode` to n fp32 offsets with the same device
  * function the fused kernel uses (Eq. m-exact / Eq. rowmax-pot / Eq. h15; the h15 input is clamped
- * below at -126, App. B.1 "Implementation").  x and w are device arrays of n floats; they may alias.
+ * below at -126, App. B.1 "Implementation"; inside the fused kernel a key tile that holds masked scores
+ * clamps at -127 instead, the input whose weight pattern is +0, so that a masked key weighs nothing).  x and w are device arrays of n floats; they may alias.
  * pot and h15 results are bit-exact by definition; exact uses the hardware ex2 approximation with
  * subnormal results flushed to zero.
  */
