@@ -6,15 +6,15 @@
 //   x = s*c - m*c -> weight map -> row sum l and P (same weights) -> O = alpha*O + P V;
 // at the end O = v_descale * O / l and LSE = ln2 * (m*c + log2 l).
 //
-// One CTA (16 warps) owns two query tiles of 128 rows of one (batch, head) and walks their key
-// tiles once, so every K/V tile staged in shared memory feeds four MMAs:
+// Persistent grid: one CTA (16 warps) per SM walks work items, each a pair of query tiles of 128 rows
+// of one (batch, head) whose key tiles it visits once, so every K/V tile staged in shared memory
+// feeds four MMAs:
 //   warpgroup 0/1  softmax of query tile 0/1: one thread per row (no shuffles needed: a thread
 //                  reads its whole score row from TMEM), weight map, row sum, P written back to
-//                  TMEM over the S columns
-//   warpgroup 2    correction: rescales the O accumulators in TMEM when a running maximum moved,
-//                  and runs the epilogue
+//                  TMEM over the S columns; after the last key tile the epilogue of its rows
+//   warpgroup 2    correction: rescales the O accumulators in TMEM when a running maximum moved
 //   warp 12        MMA issuer (one thread): S_t = Q_t K^T and O_t += P_t V on the tensor cores
-//   warp 13        TMA producer (one thread): Q once, then K/V through a ring of shared-memory slots
+//   warp 13        TMA producer (one thread): Q per item, K/V through a ring of shared-memory slots
 // While warpgroup 0 works on S_0(j), the tensor cores compute P_1 V(j-1) and S_1(j), and vice versa.
 // TMEM columns: S_0/P_0 [0,128), S_1/P_1 [128,256), O_0 [256,384), O_1 [384,512).
 #include "softmax_math.cuh"
