@@ -24,8 +24,12 @@
  * the unshifted Schraudolph construction on half-integer-rounded inputs; the add-and-shift bit
  * construction; brute-force and library softmax on tiny inputs; Q = 0 closed form; two-key hand
  * example; whole-row equivalence when one tile covers the row; a second, independent NumPy coding
- * of the online loop.  Parity unpinned: the tie-widening rule (oracle_attn's widen outputs) and the
- * p_round diagnostic are this build's own devices and have no counterpart in the paper.
+ * of the online loop; with a rescale threshold: exact mode equals the definition for any threshold,
+ * and a hand example with a lagging anchor (positive offsets); Rowmax-PoT tail: clamp and drop values
+ * at and beyond K_max.  The tie-widening rule (oracle_attn's widen outputs) and the p_round diagnostic
+ * are this build's own devices with no counterpart in the paper; they are pinned as what they claim
+ * to be: p_round against a library's casts to bfloat16 / e4m3 / e5m2, the widening as a bound, by
+ * moving every flagged score across its boundary.
  */
 #include <fenv.h>
 #include <math.h>
@@ -95,7 +99,7 @@ double oracle_decode_e4m3(uint8_t b) {
 
 /* Round a non-negative double to a format with `fbits` fraction bits, minimum normal exponent
  * `emin` and largest finite value `vmax`, ties to even, saturating.  Used only by the p_round
- * diagnostic below. */
+ * diagnostic below (pinned in the tests against a library's casts to bfloat16, e4m3 and e5m2). */
 static double round_to_small_float(double v, int fbits, int emin, double vmax) {
     if (!(v > 0.0)) return 0.0;
     int e;
@@ -119,6 +123,10 @@ static double p_round_apply(double w, int p_round, int p_off) {
     return ldexp(r, -p_off);
 }
 
+/* The p_round diagnostic on one value, exported so that tests can pin it:
+ * the weight w >= 0 times 2^p_off rounded to the format, divided by 2^p_off again. */
+double oracle_p_round(double w, int p_round, int p_off) { return p_round_apply(w, p_round, p_off); }
+
 /* ---------------------------------------------------------------------------------------------
  * Weight maps on an fp32 base-two offset x (x = 0 at the anchor, negative below it).
  * ------------------------------------------------------------------------------------------- */
@@ -127,14 +135,20 @@ static double p_round_apply(double w, int p_round, int p_off) {
 double oracle_w_exact(float x) { return exp2((double)x); }
 
 /* Rowmax-PoT (Eq. rowmax-pot): with y = Delta/ln2 = -x, d = min{K_max, floor(y + 1/2)}, w = 2^-d.
- * Ties in y + 1/2 go up in d, that is toward the smaller weight. */
-double oracle_w_pot(float x, int kmax) {
+ * Ties in y + 1/2 go up in d, that is toward the smaller weight.  The main point clamps the tail
+ * (every key keeps at least 2^-K_max: full support); the tail-drop variant (App. A, the sentence
+ * after Eq. rowmax-pot) gives weight zero to the keys whose index floor(y + 1/2) exceeds K_max. */
+double oracle_w_pot_tail(float x, int kmax, int drop_tail) {
     if (isnan(x)) return NAN;
     double y = -(double)x;
     double d = floor(y + 0.5); /* exact: y is an fp32 value, the sum is representable in double */
-    if (d > (double)kmax) d = (double)kmax;
+    if (d > (double)kmax) {
+        if (drop_tail) return 0.0;
+        d = (double)kmax;
+    }
     return ldexp(1.0, -(int)d);
 }
+double oracle_w_pot(float x, int kmax) { return oracle_w_pot_tail(x, kmax, 0); }
 
 /* Rowmax-H15 (Eq. h15): n = RNE(2x), w = (1 + (n mod 2)/2) * 2^floor(n/2), floor toward -inf and
  * n mod 2 the non-negative residue; the input is first clamped from below at -126 (the doubled
@@ -163,9 +177,9 @@ double oracle_w_h15_family(float x, int k) {
     return ldexp(1.0 + (q - fl), (int)fl);
 }
 
-static double weight_of(float x, int mode, int kmax) {
+static double weight_of(float x, int mode, int kmax, int drop_tail) {
     switch (mode) {
-        case ORACLE_W_POT: return oracle_w_pot(x, kmax);
+        case ORACLE_W_POT: return oracle_w_pot_tail(x, kmax, drop_tail);
         case ORACLE_W_H15: return oracle_w_h15(x);
         case ORACLE_W_H15K2: return oracle_w_h15_family(x, 2);
         case ORACLE_W_H15K3: return oracle_w_h15_family(x, 3);
@@ -174,10 +188,10 @@ static double weight_of(float x, int mode, int kmax) {
 }
 
 /* Array form used by the sweep tests.  Returns 0, or -1 for a bad mode. */
-int oracle_weight_map(const float* x, double* w, size_t n, int mode, int kmax) {
+int oracle_weight_map(const float* x, double* w, size_t n, int mode, int kmax, int drop_tail) {
     if (mode < 0 || mode > 4) return -1;
     fesetround(FE_TONEAREST);
-    for (size_t i = 0; i < n; ++i) w[i] = weight_of(x[i], mode, kmax);
+    for (size_t i = 0; i < n; ++i) w[i] = weight_of(x[i], mode, kmax, drop_tail);
     return 0;
 }
 
@@ -257,12 +271,12 @@ static void row_exact_definition(const double* qrow, const double* kbase, const 
  * its tolerance on exactly those rows. */
 static void row_online(const double* qrow, const double* kbase, const double* vbase,
                        size_t kv_stride, int nvis, int D, float c32, double dv, int mode,
-                       int tile_n, int kv_order, double tau, int kmax, int p_round, int p_off,
-                       double tie_eps, double* z_buf, double* o, double* lse, double* widen_o,
+                       int tile_n, int kv_order, double tau, int kmax, int drop_tail, int p_round,
+                       int p_off, double tie_eps, double* z_buf, double* o, double* lse, double* widen_o,
                        double* widen_lse, int32_t* nflag) {
     double c = (double)c32;
     double m = -INFINITY, l = 0.0;
-    double flip = 0.0, flip_vmax = 0.0;
+    double flip = 0.0, flip_down = 0.0, flip_vmax = 0.0;
     int32_t flagged = 0;
     for (int d = 0; d < D; ++d) o[d] = 0.0;
     if (nvis <= 0) {
@@ -290,13 +304,14 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
             double alpha = (m == -INFINITY) ? 0.0 : exp2((m - m_new) * c);
             l *= alpha;
             flip *= alpha;
+            flip_down *= alpha;
             for (int d = 0; d < D; ++d) o[d] *= alpha;
             m = m_new;
         }
         double mc = (double)(float)(m * c);
         for (int j = j0; j < j1; ++j) {
             float x = (float)(z_buf[j - j0] * c - mc);
-            double w = weight_of(x, mode, kmax);
+            double w = weight_of(x, mode, kmax, drop_tail);
             const double* vr = vbase + (size_t)j * kv_stride;
             double pw = p_round_apply(w, p_round, p_off);
             l += w;
@@ -315,7 +330,11 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
                     double vmax = 0.0;
                     for (int d = 0; d < D; ++d)
                         if (fabs(vr[d]) > vmax) vmax = fabs(vr[d]);
-                    flip += kk > 0 ? ldexp(w, -kk) : w;   /* one lattice step is at most w / 2^k */
+                    /* one lattice step is at most w / 2^k (pot: w; a dropped tail weight may come back as 2^-K_max) */
+                    flip += kk > 0 ? ldexp(w, -kk) : (w > 0.0 ? w : ldexp(1.0, -kmax));
+                    /* the largest step DOWN is w / (2^k + 1) (from (1 + 2^-k) 2^e to 2^e; pot: w / 2); a
+                     * tail weight 2^-K_max that is dropped loses all of itself */
+                    flip_down += (kk == 0 && drop_tail && w <= ldexp(1.0, -kmax)) ? w : w / (ldexp(1.0, kk) + 1.0);
                     if (vmax > flip_vmax) flip_vmax = vmax;
                     ++flagged;
                 }
@@ -328,7 +347,8 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
         if (fabs(o[d]) > omax) omax = fabs(o[d]);
     }
     *lse = M_LN2 * (m * c + log2(l));
-    if (widen_o) *widen_o = (flip / l) * (dv * flip_vmax + omax);
+    /* O' - O = sum_j delta_j (dv v_j - O) / l' with l' = l + sum_j delta_j >= l - flip_down */
+    if (widen_o) *widen_o = (flip / (l - flip_down)) * (dv * flip_vmax + omax);
     if (widen_lse) *widen_lse = flip / l;
     if (nflag) *nflag = flagged;
 }
@@ -341,6 +361,7 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
  *               > 0 = the online loop with tiles of tile_n keys (any mode)
  *   kv_order    +1 ascending key tiles, -1 descending
  *   tau         rescale threshold in octaves (0 = always rescale)
+ *   kmax, drop_tail   Rowmax-PoT: tail index K_max and what happens beyond it (0 = clamp, 1 = drop)
  *   p_round     diagnostic only: round the weight (times 2^p_off) to bf16 / e4m3 / e5m2 before it
  *               multiplies V; the row sum always uses the unrounded weight
  *   tie_eps     0 disables the tie bookkeeping; widen_o, widen_lse, nflag may be NULL
@@ -349,7 +370,7 @@ static void row_online(const double* qrow, const double* kbase, const double* vb
 int oracle_attn(const void* q, const void* k, const void* v, int in_dtype, int B, int Hq, int Hkv,
                 int Sq, int Sk, int D, int causal, float softmax_scale, float q_descale,
                 float k_descale, float v_descale, int mode, int tile_n, int kv_order, double tau,
-                int kmax, int p_round, int p_off, double tie_eps, const int32_t* rows, int nrows,
+                int kmax, int drop_tail, int p_round, int p_off, double tie_eps, const int32_t* rows, int nrows,
                 double* O, double* LSE, double* widen_o, double* widen_lse, int32_t* nflag,
                 int nthreads) {
     if (!q || !k || !v || !O || !LSE) return -1;
@@ -409,7 +430,8 @@ int oracle_attn(const void* q, const void* k, const void* v, int in_dtype, int B
                 if (nflag) nflag[it] = 0;
             } else {
                 row_online(qrow, kbase, vbase, kv_stride, nvis, D, c32, dv, mode, tile_n,
-                           kv_order, tau, kmax, p_round, p_off, tie_eps, buf, o, LSE + it,
+                           kv_order, tau, kmax, drop_tail, p_round, p_off, tie_eps, buf, o,
+                           LSE + it,
                            widen_o ? widen_o + it : NULL, widen_lse ? widen_lse + it : NULL,
                            nflag ? nflag + it : NULL);
             }

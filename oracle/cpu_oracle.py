@@ -47,11 +47,13 @@ def lib() -> ctypes.CDLL:
         L.oracle_decode_e4m3.argtypes = [ctypes.c_uint8]
         L.oracle_weight_map.restype = ctypes.c_int
         L.oracle_weight_map.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
-                                        ctypes.c_int, ctypes.c_int]
+                                        ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.oracle_p_round.restype = ctypes.c_double
+        L.oracle_p_round.argtypes = [ctypes.c_double, ctypes.c_int, ctypes.c_int]
         L.oracle_attn.restype = ctypes.c_int
         L.oracle_attn.argtypes = (
             [ctypes.c_void_p] * 3 + [ctypes.c_int] * 8 + [ctypes.c_float] * 4
-            + [ctypes.c_int] * 3 + [ctypes.c_double] + [ctypes.c_int] * 3 + [ctypes.c_double]
+            + [ctypes.c_int] * 3 + [ctypes.c_double] + [ctypes.c_int] * 4 + [ctypes.c_double]
             + [ctypes.c_void_p, ctypes.c_int] + [ctypes.c_void_p] * 5 + [ctypes.c_int])
         _lib = L
     return _lib
@@ -69,18 +71,23 @@ def decode_e4m3(bits: int) -> float:
     return lib().oracle_decode_e4m3(int(bits))
 
 
-def weight_map(x, mode: int, kmax: int = 20) -> np.ndarray:
-    """Weights (float64) of the fp32 offsets ``x`` under ``mode``."""
+def p_round(w: float, fmt: int, p_off: int = 0) -> float:
+    """The P-storage diagnostic on one weight: w * 2^p_off rounded to ``fmt``, divided by 2^p_off."""
+    return lib().oracle_p_round(float(w), fmt, p_off)
+
+
+def weight_map(x, mode: int, kmax: int = 20, drop_tail: bool = False) -> np.ndarray:
+    """Weights (float64) of the fp32 offsets ``x`` under ``mode`` (``kmax``, ``drop_tail``: Rowmax-PoT only)."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     w = np.empty(x.shape, dtype=np.float64)
-    rc = lib().oracle_weight_map(x.ctypes.data, w.ctypes.data, x.size, mode, kmax)
+    rc = lib().oracle_weight_map(x.ctypes.data, w.ctypes.data, x.size, mode, kmax, int(drop_tail))
     if rc != 0:
         raise ValueError(f"oracle_weight_map failed: {rc}")
     return w
 
 
 def attn(q, k, v, *, in_dtype: int, causal: bool, softmax_scale: float, mode: int,
-         tile_n: int = 0, kv_order: int = 1, tau: float = 0.0, kmax: int = 20,
+         tile_n: int = 0, kv_order: int = 1, tau: float = 0.0, kmax: int = 20, drop_tail: bool = False,
          q_descale: float = 1.0, k_descale: float = 1.0, v_descale: float = 1.0,
          p_round: int = P_NONE, p_off: int = 0, tie_eps: float = 0.0, rows=None,
          nthreads: int = 0):
@@ -111,7 +118,8 @@ def attn(q, k, v, *, in_dtype: int, causal: bool, softmax_scale: float, mode: in
     nflag = np.zeros((B, Hq, nrows), dtype=np.int32)
     rc = lib().oracle_attn(q.ctypes.data, k.ctypes.data, v.ctypes.data, in_dtype, B, Hq, Hkv, Sq,
                            Sk, D, int(bool(causal)), softmax_scale, q_descale, k_descale,
-                           v_descale, mode, tile_n, kv_order, float(tau), kmax, p_round, p_off,
+                           v_descale, mode, tile_n, kv_order, float(tau), kmax, int(drop_tail), p_round,
+                           p_off,
                            float(tie_eps), rows_ptr, nrows, O.ctypes.data, LSE.ctypes.data,
                            widen_o.ctypes.data, widen_lse.ctypes.data, nflag.ctypes.data, nthreads)
     if rc < 0:

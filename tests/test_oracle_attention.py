@@ -147,9 +147,10 @@ def test_two_key_hand_example():
 
 # ---- a second, independent coding of the online loop -------------------------------------------
 
-def _numpy_online(q, k, v, causal, scale, mode, tile_n, order=1, tau=0.0, kmax=20):
+def _numpy_online(q, k, v, causal, scale, mode, tile_n, order=1, tau=0.0, kmax=20, drop_tail=False, reweigh=None):
     """NumPy restatement of the online loop (running maximum per key tile, rescale, shared weights
-    for the row sum and PV), vectorised over the tile and coded separately from the C oracle."""
+    for the row sum and PV), vectorised over the tile and coded separately from the C oracle.
+    `reweigh(x32, w)` may replace the weights of a tile (used to move scores across a rounding boundary)."""
     B, Sq, Hq, D = q.shape
     Sk, Hkv = k.shape[1], k.shape[2]
     c = np.float32(scale * LOG2E)
@@ -161,7 +162,8 @@ def _numpy_online(q, k, v, causal, scale, mode, tile_n, order=1, tau=0.0, kmax=2
         if mode == orc.W_EXACT:
             return np.exp2(x)
         if mode == orc.W_POT:
-            return np.exp2(-np.minimum(kmax, np.floor(-x + 0.5)))
+            d = np.floor(-x + 0.5)
+            return np.where((d > kmax) & drop_tail, 0.0, np.exp2(-np.minimum(kmax, d)))
         if mode in (orc.W_H15K2, orc.W_H15K3):
             st = 4.0 if mode == orc.W_H15K2 else 8.0
             q = np.rint(st * np.maximum(x, -126.0)) / st
@@ -188,7 +190,10 @@ def _numpy_online(q, k, v, causal, scale, mode, tile_n, order=1, tau=0.0, kmax=2
                         alpha = 0.0 if m == -np.inf else 2.0 ** ((m - mn) * cd)
                         l *= alpha; acc *= alpha; m = mn
                     mc = float(np.float32(m * cd))
-                    w = wmap((z[a:e] * cd - mc).astype(np.float32))
+                    x32 = (z[a:e] * cd - mc).astype(np.float32)
+                    w = wmap(x32)
+                    if reweigh is not None:
+                        w = reweigh(x32, w, wmap)
                     l += w.sum(); acc += w @ v[b, a:e, hk]
                 O[b, h, i] = acc / l
                 L[b, h, i] = math.log(2.0) * (m * cd + math.log2(l))
@@ -205,6 +210,48 @@ def test_online_matches_independent_numpy_coding(mode, tile_n, order, tau):
     got = _run(wl, mode, tile_n, inp, kv_order=order, tau=tau)
     assert np.allclose(got["O"], O, rtol=1e-11, atol=1e-12)
     assert np.allclose(got["LSE"], L, rtol=1e-11, atol=1e-12)
+
+
+# ---- the deferred rescale (threshold tau > 0) against what the mathematics fixes ----------------
+
+@pytest.mark.parametrize("tau", [2.0, 8.0])
+@pytest.mark.parametrize("tile_n", [8, 16, 128])
+def test_exact_mode_does_not_depend_on_the_rescale_threshold(tau, tile_n):
+    # With w = 2^x the anchor cancels between numerator and denominator: any adoption rule gives the
+    # softmax of the definition, in O and in LSE.
+    for wl in (TINY_X, SMALL):
+        inp = make_inputs(wl)
+        want = _run(wl, orc.W_EXACT, 0, inp)
+        got = _run(wl, orc.W_EXACT, tile_n, inp, tau=tau)
+        assert np.allclose(got["O"], want["O"], rtol=0, atol=2e-7)      # x is rounded to fp32 in the loop
+        assert np.allclose(got["LSE"], want["LSE"], rtol=0, atol=2e-6)
+
+
+def test_lagging_anchor_hand_example():
+    # One query, four keys, tiles of ONE key, c = 1, tau = 1.  Scores 0, 0.5, 1, 3 octaves.
+    #   key 0: first tile, anchor m = 0, x = 0                      -> every map gives 1
+    #   key 1: 0.5 above the anchor, not more than tau: m stays 0, x = +0.5
+    #          h15: n = RNE(1) = 1 -> 1.5 (Eq. h15 covers positive x); pot: floor(-0.5 + 0.5) = 0 -> 1; exact: 2^0.5
+    #   key 2: 1.0 above, still not MORE than tau: x = +1 -> h15 2, pot 2^-floor(-0.5) = 2, exact 2
+    #   key 3: 3.0 above > tau: adopted, alpha = 2^-3, x = 0 -> 1
+    D = 8
+    q = np.zeros((1, 1, 1, D), np.float32); q[..., 0] = 1.0
+    k = np.zeros((1, 4, 1, D), np.float32); k[0, :, 0, 0] = [0.0, 0.5, 1.0, 3.0]
+    v = np.zeros((1, 4, 1, D), np.float32); v[0, :, 0, 0] = [1.0, -2.0, 4.0, 8.0]; v[0, :, 0, 1] = 1.0
+    scale = float(np.float32(math.log(2.0)))       # c = fl32(ln2 * log2 e) = 1 exactly
+    for mode, w1, w2 in ((orc.W_H15, 1.5, 2.0), (orc.W_POT, 1.0, 2.0), (orc.W_EXACT, 2.0 ** 0.5, 2.0)):
+        got = orc.attn(_bf16_bits(q), _bf16_bits(k), _bf16_bits(v), in_dtype=orc.IN_BF16, causal=False,
+                       softmax_scale=scale, mode=mode, tile_n=1, tau=1.0)
+        l = (1.0 + w1 + w2) / 8.0 + 1.0
+        want0 = ((1.0 * 1.0 + w1 * -2.0 + w2 * 4.0) / 8.0 + 8.0) / l
+        assert abs(got["O"][0, 0, 0, 0] - want0) < 1e-12, (mode, got["O"][0, 0, 0, 0], want0)
+        assert abs(got["O"][0, 0, 0, 1] - 1.0) < 1e-12
+        assert abs(got["LSE"][0, 0, 0] - math.log(2.0) * (3.0 + math.log2(l))) < 1e-12
+    # tau = 0 on the same input: every tile is adopted, every x is 0, the rescales carry the differences
+    got = orc.attn(_bf16_bits(q), _bf16_bits(k), _bf16_bits(v), in_dtype=orc.IN_BF16, causal=False,
+                   softmax_scale=scale, mode=orc.W_H15, tile_n=1, tau=0.0)
+    l = ((1.0 * 2.0 ** -0.5 + 1.0) * 2.0 ** -0.5 + 1.0) * 0.25 + 1.0
+    assert abs(got["LSE"][0, 0, 0] - math.log(2.0) * (3.0 + math.log2(l))) < 1e-12
 
 
 # ---- equivalences fixed by the mathematics -----------------------------------------------------

@@ -173,6 +173,29 @@ def test_pot_properties():
         assert orc.weight_map(np.array([xv], np.float32), orc.W_POT)[0] == 2.0 ** -dd
 
 
+@pytest.mark.parametrize("kmax", [8, 12, 20, 48])
+def test_pot_tail_clamp_and_drop(kmax):
+    # App. A, after Eq. rowmax-pot: the main point clamps the tail at K_max (full support); the tail-drop
+    # variant removes the keys whose index exceeds K_max.  Index d = floor(y + 1/2), y = -x.
+    x = inputs.weight_map_sweep()
+    x = x[np.isfinite(x) & (x <= 0)]
+    clamp = orc.weight_map(x, orc.W_POT, kmax=kmax)
+    drop = orc.weight_map(x, orc.W_POT, kmax=kmax, drop_tail=True)
+    d = np.floor(-x.astype(np.float64) + 0.5)
+    assert np.array_equal(clamp, 2.0 ** -np.minimum(d, kmax))
+    assert np.array_equal(drop, np.where(d > kmax, 0.0, 2.0 ** -d))
+    assert np.array_equal(clamp[d <= kmax], drop[d <= kmax])            # the two agree on the body
+    one = lambda v, **kw: orc.weight_map(np.array([v], np.float32), orc.W_POT, kmax=kmax, **kw)[0]   # noqa: E731
+    assert one(-(kmax + 1)) == 2.0 ** -kmax and one(-(kmax + 1), drop_tail=True) == 0.0
+    assert one(-kmax) == 2.0 ** -kmax == one(-kmax, drop_tail=True)
+    assert one(-(kmax + 0.5), drop_tail=True) == 0.0                     # ties go up in d: d = K_max + 1 is dropped
+    assert one(np.nextafter(np.float32(-(kmax + 0.5)), np.float32(0)), drop_tail=True) == 2.0 ** -kmax
+    assert one(-np.inf) == 2.0 ** -kmax and one(-np.inf, drop_tail=True) == 0.0
+    order = np.argsort(x, kind="stable")
+    assert np.all(np.diff(clamp[order]) >= 0) and np.all(np.diff(drop[order]) >= 0)   # both monotone
+    assert one(0.0) == 1.0 == one(0.0, drop_tail=True)
+
+
 def test_pot_no_double_rounding_at_fp32_edge():
     # y = 0.5 - 2^-25 is an fp32 value; y + 0.5 rounds to 1.0 in fp32 but floor(y + 1/2) is 0.
     x = np.float32(-(0.5 - 2.0 ** -25))
