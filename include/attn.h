@@ -23,8 +23,9 @@
  *     frees or keeps them.  Calls are asynchronous on `stream` (a cudaStream_t passed as void*;
  *     NULL = the legacy default stream) and do not synchronise the host.
  *   - Return value: ATTN_OK (0) or a negative ATTN_ERR_* code.  Nothing is thrown, printed or aborted.
- *   - Not thread-safe with respect to the per-process caches of tensor maps: call from one host
- *     thread at a time.
+ *   - The library keeps a little per-process state without locks (the address of each device's status
+ *     word, the code of the last failing CUDA call, per-device launch set-up): call from one host thread
+ *     at a time.
  */
 #ifndef ROWMAX_ATTN_H_
 #define ROWMAX_ATTN_H_
@@ -42,6 +43,11 @@ enum { ATTN_IN_BF16 = 0, ATTN_IN_FP8_E4M3 = 1, ATTN_IN_FP16 = 2 };
 /* format of the probability tile P fed to the P.V contraction, as reported by attn_get_schedule */
 enum { ATTN_P_BF16 = 0, ATTN_P_E4M3 = 1, ATTN_P_E5M2 = 2, ATTN_P_FP16 = 3 };
 
+/* Rowmax-PoT tail index K_max: default (the paper's main point) and the largest value whose weights the
+ * format of P still holds exactly (bf16: the fp32 exponent range; fp16 P: down to its subnormals; fp8:
+ * e5m2 P with a power-of-two offset, 29 octaves). */
+enum { ATTN_POT_KMAX_DEFAULT = 20, ATTN_POT_KMAX_BF16 = 125, ATTN_POT_KMAX_FP16 = 23, ATTN_POT_KMAX_FP8 = 29 };
+
 enum {
     ATTN_OK = 0,
     ATTN_ERR_NULLPTR = -1,          /* a required pointer is NULL */
@@ -52,7 +58,7 @@ enum {
     ATTN_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed; see attn_last_cuda_error */
     ATTN_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired; see attn_device_status */
     ATTN_ERR_UNSUPPORTED = -8,      /* valid arguments, combination not built (e.g. a deferred rescale on fp8 inputs) */
-    ATTN_ERR_BAD_VALUE = -9         /* softmax_scale or an fp8 descale is not positive and finite */
+    ATTN_ERR_BAD_VALUE = -9         /* softmax_scale or an fp8 descale not positive and finite; rescale_tau or K_max out of range */
 };
 
 /*
@@ -96,6 +102,22 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
                  float q_descale, float k_descale, float v_descale, float rescale_tau, void* stream);
 
 /*
+ * attn_fwd_pot — attn_fwd in Rowmax-PoT mode with the tail chosen by the caller (App. A, Eq. rowmax-pot and the
+ * sentence after it: the main point clamps the tail at K_max = 20, a K_max sweep and a tail-drop variant are
+ * reported beside it; results figure, panel B).  The index of a key is d = min{K_max, floor(-x + 1/2)} and its
+ * weight 2^-d (clamped tail, drop_tail = 0: every visible key keeps at least 2^-K_max), or, with drop_tail != 0,
+ * d = floor(-x + 1/2) and weight 0 where d > K_max.  x is the offset from the running maximum of the online
+ * loop, so with a dropped tail a key is dropped relative to the anchor of its own key tile; what earlier tiles
+ * accumulated is rescaled, not dropped.  1 <= pot_kmax <= ATTN_POT_KMAX_BF16 / _FP16 / _FP8 for the storage type,
+ * else ATTN_ERR_BAD_VALUE.  attn_fwd(..., ATTN_W_POT, ...) is attn_fwd_pot with pot_kmax = 20, drop_tail = 0.
+ */
+int attn_fwd_pot(const void* q, const void* k, const void* v, void* o, float* lse,
+                 int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                 int causal, float softmax_scale, int in_dtype,
+                 float q_descale, float k_descale, float v_descale,
+                 int pot_kmax, int drop_tail, void* stream);
+
+/*
  * attn_weight_map — applies the weight map of `weight_mode` to n fp32 offsets with the same device
  * function the fused kernel uses (Eq. m-exact / Eq. rowmax-pot / Eq. h15; the h15 input is clamped
  * below at -126, App. B.1 "Implementation"; inside the fused kernel a key tile that holds masked scores
@@ -106,6 +128,28 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
 int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* stream);
 
 /*
+ * attn_weight_map_pot — the Rowmax-PoT map with the tail of attn_fwd_pot (Eq. rowmax-pot and the sentence after
+ * it): w = 2^-min{K_max, floor(-x + 1/2)}, or with drop_tail != 0 zero where floor(-x + 1/2) > K_max.  Bit-exact
+ * by definition.  1 <= pot_kmax <= ATTN_POT_KMAX_BF16, else ATTN_ERR_BAD_VALUE.
+ */
+int attn_weight_map_pot(const float* x, float* w, size_t n, int pot_kmax, int drop_tail, void* stream);
+
+/*
+ * attn_weight_map_fused — the weights as the hot loop of attn_fwd produces them and stores them in P for inputs of
+ * storage type in_dtype (Eq. m-exact / Eq. rowmax-pot / Eq. h15 again, but through the instantiations the fused
+ * kernel runs, which attn_weight_map does not reach: the h15 family without the per-score clamp wherever 32
+ * consecutive offsets all lie above -125 octaves, with the clamp elsewhere; weights scaled by the P offset;
+ * Rowmax-PoT evaluated on the negated offset, with the tail given here).  The n offsets are taken 32 at a time as
+ * one chunk of a score row; the packed P words are decoded again and divided by the P scale.  For the lattice
+ * maps the result equals attn_weight_map bit for bit wherever P can hold the weight: everywhere for bf16 P, down
+ * to 2^-23 for fp16 P (powers of two: 2^-24), down to 2^-29 for e5m2 P (pot, h15, h15k2 on fp8 inputs) and down to 2^-14
+ * for e4m3 P (h15k3 on fp8 inputs); below that P underflows towards zero.  exact-like modes are rounded to the
+ * format of P.  pot_kmax / drop_tail matter in ATTN_W_POT mode only (limits as for attn_fwd_pot).
+ */
+int attn_weight_map_fused(const float* x, float* w, size_t n, int weight_mode, int in_dtype,
+                          int pot_kmax, int drop_tail, void* stream);
+
+/*
  * attn_get_schedule — what a reference implementation must mirror to reproduce pot/h15 results
  * (App. B "Semantic simulation": per-tile running maximum, tile of 128 keys, rescale rule).
  * Host-only query, no CUDA call.  Any output pointer may be NULL.
@@ -113,7 +157,7 @@ int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* s
  *   kv_order         +1: key tiles visited in ascending order
  *   rescale_tau      anchor adoption threshold in octaves used by attn_fwd (0 = the anchor is always current);
  *                    attn_fwd_tau takes its own
- *   pot_kmax         K_max of Rowmax-PoT
+ *   pot_kmax         K_max of Rowmax-PoT as attn_fwd uses it (attn_fwd_pot takes its own)
  *   p_format         ATTN_P_*; p_offset_log2: P is stored as weight * 2^p_offset_log2
  */
 int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal,

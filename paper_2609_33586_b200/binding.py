@@ -20,7 +20,7 @@ MODES = {"exact": W_EXACT, "pot": W_POT, "h15": W_H15, "h15k2": W_H15K2, "h15k3"
 _LIB_PATH = Path(__file__).resolve().parent / "libattn_b200.so"
 _lib = None
 
-EXPORTS = ("attn_fwd", "attn_fwd_tau", "attn_weight_map", "attn_get_schedule", "attn_device_status",
+EXPORTS = ("attn_fwd", "attn_fwd_tau", "attn_fwd_pot", "attn_weight_map", "attn_weight_map_pot", "attn_weight_map_fused", "attn_get_schedule", "attn_device_status",
            "attn_device_status_reset", "attn_launch_count", "attn_status_string",
            "attn_last_cuda_error", "attn_version")
 
@@ -44,8 +44,14 @@ def lib() -> ctypes.CDLL:
         L.attn_fwd.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, f, f, f, vp]
         L.attn_fwd_tau.restype = i
         L.attn_fwd_tau.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, f, f, f, f, vp]
+        L.attn_fwd_pot.restype = i
+        L.attn_fwd_pot.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, f, f, f, i, i, vp]
         L.attn_weight_map.restype = i
         L.attn_weight_map.argtypes = [vp, vp, ctypes.c_size_t, i, vp]
+        L.attn_weight_map_pot.restype = i
+        L.attn_weight_map_pot.argtypes = [vp, vp, ctypes.c_size_t, i, i, vp]
+        L.attn_weight_map_fused.restype = i
+        L.attn_weight_map_fused.argtypes = [vp, vp, ctypes.c_size_t, i, i, i, i, vp]
         L.attn_get_schedule.restype = i
         L.attn_get_schedule.argtypes = [i, i, i, i] + [vp] * 7
         L.attn_device_status.restype = i
@@ -111,9 +117,14 @@ def in_dtype_of(t: torch.Tensor) -> int:
 
 
 def attn_fwd_raw(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale,
-                 weight_mode, in_dtype, q_descale, k_descale, v_descale, stream_ptr, rescale_tau=None) -> int:
+                 weight_mode, in_dtype, q_descale, k_descale, v_descale, stream_ptr, rescale_tau=None,
+                 pot_tail=None) -> int:
     """Direct call with integer device addresses; returns the status code.  With `rescale_tau` the
-    call goes to attn_fwd_tau."""
+    call goes to attn_fwd_tau, with `pot_tail` = (K_max, drop_tail) to attn_fwd_pot."""
+    if pot_tail is not None:
+        return lib().attn_fwd_pot(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
+                                  softmax_scale, in_dtype, q_descale, k_descale, v_descale,
+                                  int(pot_tail[0]), int(bool(pot_tail[1])), stream_ptr)
     if rescale_tau is None:
         return lib().attn_fwd(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
                               softmax_scale, weight_mode, in_dtype, q_descale, k_descale, v_descale,
@@ -126,10 +137,13 @@ def attn_fwd_raw(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, cau
 def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool, softmax_scale: float,
              weight_mode: int, q_descale: float = 1.0, k_descale: float = 1.0, v_descale: float = 1.0,
              out: torch.Tensor | None = None, lse: torch.Tensor | None = None, return_lse: bool = True,
-             rescale_tau: float | None = None, stream=None):
+             rescale_tau: float | None = None, pot_tail=None, stream=None):
     """q (B,Sq,Hq,D), k/v (B,Sk,Hkv,D): contiguous CUDA tensors, bf16, float16 or float8_e4m3fn.
     Returns (O bf16 (B,Sq,Hq,D), LSE fp32 (B,Hq,Sq) or None).  `rescale_tau` (bf16 inputs only) selects
-    the deferred-rescale entry point attn_fwd_tau."""
+    the deferred-rescale entry point attn_fwd_tau; `pot_tail` = (K_max, drop_tail) selects attn_fwd_pot
+    (Rowmax-PoT with that tail; `weight_mode` must then be W_POT)."""
+    if pot_tail is not None and weight_mode != W_POT:
+        raise ValueError("pot_tail goes with weight_mode = W_POT")
     for t in (q, k, v):
         if not t.is_cuda or not t.is_contiguous():
             raise ValueError("q, k, v must be contiguous CUDA tensors")
@@ -147,7 +161,7 @@ def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool,
     rc = attn_fwd_raw(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                       lse.data_ptr() if lse is not None else None, B, Hq, Hkv, Sq, Sk, D, causal,
                       softmax_scale, weight_mode, dt, q_descale, k_descale, v_descale,
-                      _stream_ptr(stream), rescale_tau)
+                      _stream_ptr(stream), rescale_tau, pot_tail)
     if rc != 0:
         raise AttnError(rc, "attn_fwd")
     return out, lse
@@ -162,4 +176,30 @@ def weight_map(x: torch.Tensor, weight_mode: int, out: torch.Tensor | None = Non
     rc = lib().attn_weight_map(x.data_ptr(), out.data_ptr(), x.numel(), weight_mode, _stream_ptr(stream))
     if rc != 0:
         raise AttnError(rc, "attn_weight_map")
+    return out
+
+
+def weight_map_pot(x: torch.Tensor, kmax: int, drop_tail: bool, out: torch.Tensor | None = None, stream=None):
+    """Rowmax-PoT with the tail index `kmax`, clamped or dropped, on a contiguous fp32 CUDA tensor of offsets."""
+    if not x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous():
+        raise ValueError("x must be a contiguous fp32 CUDA tensor")
+    if out is None:
+        out = torch.empty_like(x)
+    rc = lib().attn_weight_map_pot(x.data_ptr(), out.data_ptr(), x.numel(), int(kmax), int(bool(drop_tail)), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_weight_map_pot")
+    return out
+
+
+def weight_map_fused(x: torch.Tensor, weight_mode: int, in_dtype: int, kmax: int = 20, drop_tail: bool = False,
+                     out: torch.Tensor | None = None, stream=None):
+    """The weights as the fused kernel's hot loop stores them in P for inputs of storage type `in_dtype`."""
+    if not x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous():
+        raise ValueError("x must be a contiguous fp32 CUDA tensor")
+    if out is None:
+        out = torch.empty_like(x)
+    rc = lib().attn_weight_map_fused(x.data_ptr(), out.data_ptr(), x.numel(), weight_mode, in_dtype, int(kmax),
+                                     int(bool(drop_tail)), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_weight_map_fused")
     return out

@@ -13,6 +13,9 @@ namespace rowmax {
 cudaError_t launch_attn_fwd(int D, int in_type, int mode, const CUtensorMap& tq, const CUtensorMap& tk,
                             const CUtensorMap& tv, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cudaStream_t stream);
+cudaError_t launch_weight_map_pot(const float* x, float* w, size_t n, int kmax, int drop, cudaStream_t stream);
+cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_cap,
+                                    float pot_drop_y, cudaStream_t stream);
 cudaError_t status_word_address(int** out);
 }  // namespace rowmax
 
@@ -116,9 +119,14 @@ void attn_set_trace(long long* device_buffer, int block) {
 }
 #endif
 
-int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
-                 int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
-                 float k_descale, float v_descale, float rescale_tau, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// Every forward entry point ends here.  pot_kmax / pot_drop_tail matter in ATTN_W_POT mode only.
+int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+             int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
+             float k_descale, float v_descale, float rescale_tau, int pot_kmax, int pot_drop_tail, void* stream) {
     if (!q || !k || !v || !o) return ATTN_ERR_NULLPTR;
     if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
     if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3 && in_dtype != ATTN_IN_FP16) return ATTN_ERR_BAD_ENUM;
@@ -137,6 +145,12 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
     if (in_dtype == ATTN_IN_FP16 && rescale_tau != 0.f) return ATTN_ERR_UNSUPPORTED;   // fp16 P: not built
     if (in_dtype == ATTN_IN_FP16 && weight_mode != ATTN_W_EXACT && weight_mode != ATTN_W_POT && weight_mode != ATTN_W_H15)
         return ATTN_ERR_UNSUPPORTED;
+    const bool drop = pot_drop_tail != 0;
+    if (weight_mode == ATTN_W_POT) {
+        // the tail index must stay inside what the format of P can hold exactly (see attn_fwd_pot in attn.h)
+        const int kmax_hi = fp8 ? ATTN_POT_KMAX_FP8 : (in_dtype == ATTN_IN_FP16 ? ATTN_POT_KMAX_FP16 : ATTN_POT_KMAX_BF16);
+        if (pot_kmax < 1 || pot_kmax > kmax_hi) return ATTN_ERR_BAD_VALUE;
+    }
     int rc = check_arch();
     if (rc != ATTN_OK) return rc;
 
@@ -152,6 +166,9 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
     p.v_descale = fp8 ? v_descale : 1.0f;
     p.two22 = 1u << 22;
     p.tau = rescale_tau;
+    p.pot_cap = static_cast<float>(pot_kmax) + (drop ? 1.25f : 0.25f);
+    p.pot_drop_y = drop ? static_cast<float>(pot_kmax) + 0.5f : INFINITY;
+
 #ifdef ROWMAX_TRACE
     p.trace = g_trace;
     p.trace_block = g_trace_block;
@@ -176,6 +193,24 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
     return ATTN_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+                 int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
+                 float k_descale, float v_descale, float rescale_tau, void* stream) {
+    return fwd_impl(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale, weight_mode, in_dtype, q_descale,
+                    k_descale, v_descale, rescale_tau, ATTN_POT_KMAX_DEFAULT, 0, stream);
+}
+
+int attn_fwd_pot(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+                 int Sk, int D, int causal, float softmax_scale, int in_dtype, float q_descale, float k_descale,
+                 float v_descale, int pot_kmax, int drop_tail, void* stream) {
+    return fwd_impl(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale, ATTN_W_POT, in_dtype, q_descale,
+                    k_descale, v_descale, 0.0f, pot_kmax, drop_tail, stream);
+}
+
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
              int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
              float k_descale, float v_descale, void* stream) {
@@ -196,6 +231,39 @@ int attn_weight_map(const float* x, float* w, size_t n, int weight_mode, void* s
     return ATTN_OK;
 }
 
+int attn_weight_map_pot(const float* x, float* w, size_t n, int pot_kmax, int drop_tail, void* stream) {
+    if (n == 0) return ATTN_OK;
+    if (!x || !w) return ATTN_ERR_NULLPTR;
+    if (pot_kmax < 1 || pot_kmax > ATTN_POT_KMAX_BF16) return ATTN_ERR_BAD_VALUE;
+    cudaError_t e = rowmax::launch_weight_map_pot(x, w, n, pot_kmax, drop_tail != 0, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return ATTN_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTN_OK;
+}
+
+int attn_weight_map_fused(const float* x, float* w, size_t n, int weight_mode, int in_dtype, int pot_kmax, int drop_tail,
+                          void* stream) {
+    if (n == 0) return ATTN_OK;
+    if (!x || !w) return ATTN_ERR_NULLPTR;
+    if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
+    if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3 && in_dtype != ATTN_IN_FP16) return ATTN_ERR_BAD_ENUM;
+    const int kmax_hi = in_dtype == ATTN_IN_FP8_E4M3 ? ATTN_POT_KMAX_FP8 : (in_dtype == ATTN_IN_FP16 ? ATTN_POT_KMAX_FP16 : ATTN_POT_KMAX_BF16);
+    if (weight_mode == ATTN_W_POT && (pot_kmax < 1 || pot_kmax > kmax_hi)) return ATTN_ERR_BAD_VALUE;
+    const bool drop = drop_tail != 0;
+    cudaError_t e = rowmax::launch_weight_map_fused(x, w, n, weight_mode, in_dtype, static_cast<float>(pot_kmax) + (drop ? 1.25f : 0.25f),
+                                                    drop ? static_cast<float>(pot_kmax) + 0.5f : INFINITY,
+                                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(e);
+        return e == cudaErrorInvalidValue ? ATTN_ERR_UNSUPPORTED : ATTN_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTN_OK;
+}
+
 int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* tile_m, int* tile_n, int* kv_order,
                       float* rescale_tau, int* pot_kmax, int* p_format, int* p_offset_log2) {
     (void)causal;
@@ -207,7 +275,7 @@ int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* til
     if (tile_n) *tile_n = rowmax::kTileN;
     if (kv_order) *kv_order = +1;
     if (rescale_tau) *rescale_tau = 0.0f;
-    if (pot_kmax) *pot_kmax = 20;
+    if (pot_kmax) *pot_kmax = ATTN_POT_KMAX_DEFAULT;
     const bool e4m3 = weight_mode == ATTN_W_EXACT || weight_mode == ATTN_W_EXACT_POLY || weight_mode == ATTN_W_H15K3;
     if (p_format) *p_format = in_dtype == ATTN_IN_FP16 ? ATTN_P_FP16 : !fp8 ? ATTN_P_BF16 : (e4m3 ? ATTN_P_E4M3 : ATTN_P_E5M2);
     if (p_offset_log2) *p_offset_log2 = !fp8 ? 0 : (e4m3 ? 8 : 15);

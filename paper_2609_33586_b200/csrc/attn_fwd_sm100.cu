@@ -455,6 +455,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 rs.c = make_float2(c_row, c_row);
                 rs.nmc = make_float2(nmc, nmc);
                 rs.two22 = p.two22;
+                rs.pot_cap = p.pot_cap;
+                rs.pot_drop_y = p.pot_drop_y;
                 rs.clamp_lo = 0.f;
                 if constexpr (kFam > 0) rs.clamp_lo = masked_tile ? h15_clamp_zero<kFam>() : h15_clamp_floor<kFam>();
                 float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -651,6 +653,114 @@ __global__ void weight_map_kernel(const float* __restrict__ x, float* __restrict
         }
         w[i] = wi;
     }
+}
+
+// Rowmax-PoT with a run-time tail (index cap K_max, clamped or dropped), the function of the 16-bit paths.
+__global__ void weight_map_pot_kernel(const float* __restrict__ x, float* __restrict__ w, size_t n, int kmax, int drop) {
+    const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride)
+        w[i] = w_pot_tail(x[i], kmax, drop != 0);
+}
+
+cudaError_t launch_weight_map_pot(const float* x, float* w, size_t n, int kmax, int drop, cudaStream_t stream) {
+    if (n == 0) return cudaSuccess;
+    size_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    weight_map_pot_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(x, w, n, kmax, drop);
+    return cudaGetLastError();
+}
+
+// The weights as the fused kernel's hot loop produces and stores them: every thread takes 32 consecutive offsets
+// as one chunk of a score row (score = offset, scale 1, anchor 0), runs weights_chunk32 with the template
+// arguments of the fused kernel for that storage type, including its choice between the unclamped and the
+// clamped h15 variant (here per chunk; in the fused kernel per warp and key tile), and decodes the packed P
+// words back to fp32, divided by the P scale.
+template <bool FP8, bool HALF, int MODE>
+__global__ void weight_map_fused_kernel(const float* __restrict__ x, float* __restrict__ w, size_t n, uint32_t two22,
+                                        float pot_cap, float pot_drop_y) {
+    constexpr int kFam = h15_family_k(MODE);
+    constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
+    const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+    for (size_t chunk = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; chunk * 32 < n; chunk += stride) {
+        uint32_t s[32];
+        float lowest = INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const size_t idx = chunk * 32 + i;
+            const float xi = idx < n ? x[idx] : 0.0f;
+            s[i] = __float_as_uint(xi);
+            lowest = fminf(lowest, xi);
+        }
+        RowScale rs;
+        const float c_row = kFam > 0 ? static_cast<float>(1 << kFam) : (MODE == kPot ? -1.0f : 1.0f);
+        const float nmc = is_exact_like(MODE) ? static_cast<float>(kOff) : 0.0f;
+        rs.c = make_float2(c_row, c_row);
+        rs.nmc = make_float2(nmc, nmc);
+        rs.two22 = two22;
+        rs.pot_cap = pot_cap;
+        rs.pot_drop_y = pot_drop_y;
+        rs.clamp_lo = 0.f;
+        if constexpr (kFam > 0) rs.clamp_lo = h15_clamp_floor<kFam>();
+        float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        uint32_t pw[16];
+        const bool clamp = kFam > 0 && !(lowest * (1 << kFam) >= -125.0f * (1 << kFam));
+        if (clamp) weights_chunk32<FP8, MODE, false, true, HALF>(s, rs, 32, acc, pw);
+        else weights_chunk32<FP8, MODE, false, false, HALF>(s, rs, 32, acc, pw);
+        const float unscale = __uint_as_float(static_cast<uint32_t>(127 - kOff) << 23);   // 2^-kOff
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            float v;
+            if constexpr (FP8) {
+                const uint32_t byte = (pw[i / 4] >> (8 * (i % 4))) & 0xFFu;
+                if constexpr (PFormat<FP8, MODE>::kE4M3) {
+                    uint32_t h2;
+                    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(static_cast<uint16_t>(byte)));
+                    v = __half2float(__ushort_as_half(static_cast<unsigned short>(h2 & 0xFFFFu)));
+                } else {
+                    v = __half2float(__ushort_as_half(static_cast<unsigned short>(byte << 8)));   // e5m2 = upper byte of fp16
+                }
+            } else {
+                const uint32_t h = (pw[i / 2] >> (16 * (i % 2))) & 0xFFFFu;
+                if constexpr (HALF) v = __half2float(__ushort_as_half(static_cast<unsigned short>(h)));
+                else v = __uint_as_float(h << 16);
+            }
+            const size_t idx = chunk * 32 + i;
+            if (idx < n) w[idx] = v * unscale;
+        }
+    }
+}
+
+template <bool FP8, bool HALF>
+static cudaError_t launch_fused_map_mode(const float* x, float* w, size_t n, int mode, float pot_cap, float pot_drop_y,
+                                         cudaStream_t stream) {
+    size_t blocks = ((n + 31) / 32 + 127) / 128;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    const unsigned g = static_cast<unsigned>(blocks);
+    switch (mode) {
+        case kExact: weight_map_fused_kernel<FP8, HALF, kExact><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+        case kPot: weight_map_fused_kernel<FP8, HALF, kPot><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+        case kH15: weight_map_fused_kernel<FP8, HALF, kH15><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+        default:
+            if constexpr (!HALF) {
+                switch (mode) {
+                    case kH15K2: weight_map_fused_kernel<FP8, HALF, kH15K2><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+                    case kH15K3: weight_map_fused_kernel<FP8, HALF, kH15K3><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+                    case kExactPoly: weight_map_fused_kernel<FP8, HALF, kExactPoly><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+                    default: return cudaErrorInvalidValue;
+                }
+            } else {
+                return cudaErrorInvalidValue;
+            }
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_cap,
+                                    float pot_drop_y, cudaStream_t stream) {
+    if (n == 0) return cudaSuccess;
+    if (in_type == kInFP8) return launch_fused_map_mode<true, false>(x, w, n, mode, pot_cap, pot_drop_y, stream);
+    if (in_type == kInFP16) return launch_fused_map_mode<false, true>(x, w, n, mode, pot_cap, pot_drop_y, stream);
+    return launch_fused_map_mode<false, false>(x, w, n, mode, pot_cap, pot_drop_y, stream);
 }
 
 cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cudaStream_t stream) {

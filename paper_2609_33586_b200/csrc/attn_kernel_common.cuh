@@ -28,6 +28,9 @@ struct AttnParams {
     float v_descale;  // 1 for bf16
     float tau;        // rescale threshold in octaves (0 = the anchor is always the running maximum)
     uint32_t two22;   // 1 << 22, kept in a register for the h15 integer multiply-add
+    // Rowmax-PoT tail (Eq. rowmax-pot and the sentence after it): index cap K_max and what happens beyond it
+    float pot_cap;    // y = -x is capped at K_max + 1/4 (clamped tail) or K_max + 1 + 1/4 (dropped tail)
+    float pot_drop_y; // dropped tail: y at or above K_max + 1/2 weighs zero; +inf with a clamped tail
     int* status;      // device-global sticky status word
 #ifdef ROWMAX_TRACE
     long long* trace;  // optional per-role cycle stamps of one CTA: [role 4][tile 64][slot 8]

@@ -176,6 +176,8 @@ struct RowScale {
     float2 nmc;    // minus the scaled anchor (plus the P offset in exact mode), both lanes
     uint32_t two22;  // 1 << 22 held in a register (see imad)
     float clamp_lo;  // h15 family, clamped variant: lower bound of the scaled offset (see w_h15_doubled_pair)
+    float pot_cap;   // pot: cap of y = -x (K_max + 1/4, or K_max + 1 + 1/4 with a dropped tail)
+    float pot_drop_y;  // pot, dropped tail: y at or above this (K_max + 1/2) weighs zero; +inf: nothing is dropped
 };
 
 // Turns 32 consecutive scores of one row into weights.  Adds them (times 2^kOffLog2) into `acc`
@@ -211,8 +213,10 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             w = w_h15_doubled_pair<kOff, CLAMP, h15_family_k(MODE)>(x, rs.two22, rs.clamp_lo);
         } else {
             // rs.c and rs.nmc carry the opposite sign in pot mode: x holds y = -(offset) >= 0
-            w.x = pot_weight_from_y<kOff>(x.x);
-            w.y = pot_weight_from_y<kOff>(x.y);
+            w.x = pot_weight_from_y<kOff>(x.x, rs.pot_cap);
+            w.y = pot_weight_from_y<kOff>(x.y, rs.pot_cap);
+            if (x.x >= rs.pot_drop_y) w.x = 0.f;
+            if (x.y >= rs.pot_drop_y) w.y = 0.f;
         }
         if constexpr (!is_exact_like(MODE) && MASKED) {
             if (2 * i >= limit) w.x = 0.f;

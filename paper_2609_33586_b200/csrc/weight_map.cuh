@@ -89,20 +89,30 @@ __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22, 
 // (offsets above the anchor occur only with a deferred rescale, whose threshold is at most 32).
 constexpr float kPotMagic = 4194368.5f;        // 2^22 + 64.5, bit pattern 0x4A800081
 constexpr uint32_t kPotMagicBase = 0x4A800000u;  // bit pattern of 2^22
-__device__ __forceinline__ uint32_t pot_tbits(float y) {
-    return __float_as_uint(__fadd_rd(fminf(y, static_cast<float>(kPotKmax) + 0.25f), kPotMagic));
+constexpr float kPotCapDefault = static_cast<float>(kPotKmax) + 0.25f;
+// `cap` = K_max + 1/4 (1 <= K_max <= 126) for the clamped tail.  For the dropped tail the callers cap at
+// K_max + 1 + 1/4, so that the index K_max + 1 survives, and give that index the weight zero.
+__device__ __forceinline__ uint32_t pot_tbits(float y, float cap = kPotCapDefault) {
+    return __float_as_uint(__fadd_rd(fminf(y, cap), kPotMagic));
 }
-__device__ __forceinline__ int pot_index_from_y(float y) {
-    return static_cast<int>((pot_tbits(y) - kPotMagicBase) >> 1) - 64;   // (2 (t - 2^22)) / 2 - 64
+__device__ __forceinline__ int pot_index_from_y(float y, float cap = kPotCapDefault) {
+    return static_cast<int>((pot_tbits(y, cap) - kPotMagicBase) >> 1) - 64;   // (2 (t - 2^22)) / 2 - 64
 }
 __device__ __forceinline__ int pot_index(float x) { return pot_index_from_y(-x); }
 // fp32 pattern of 2^(kOff - d): exponent field 127 + kOff - d = (191 + kOff) - (d + 64), and d + 64 is
 // the t pattern without its lowest bit, shifted right by one: ((tbits & ~1) << 22) puts it at bit 23
 // (the bits of 2^22's own pattern fall off the top).
 template <int kOff>
-__device__ __forceinline__ float pot_weight_from_y(float y) {
-    return __uint_as_float((static_cast<uint32_t>(191 + kOff) << 23) - ((pot_tbits(y) & ~1u) << 22));
+__device__ __forceinline__ float pot_weight_from_y(float y, float cap = kPotCapDefault) {
+    return __uint_as_float((static_cast<uint32_t>(191 + kOff) << 23) - ((pot_tbits(y, cap) & ~1u) << 22));
 }
 __device__ __forceinline__ float w_pot(float x) { return pot_weight_from_y<0>(-x); }
+// General tail: K_max as a run-time value, clamped (every key keeps 2^-K_max) or dropped (weight zero
+// beyond K_max; ties of y + 1/2 go up in the index, so y = K_max + 1/2 is already dropped).
+__device__ __forceinline__ float w_pot_tail(float x, int kmax, bool drop_tail) {
+    const float y = -x;
+    const float w = pot_weight_from_y<0>(y, static_cast<float>(kmax) + (drop_tail ? 1.25f : 0.25f));
+    return (drop_tail && y >= static_cast<float>(kmax) + 0.5f) ? 0.0f : w;
+}
 
 }  // namespace rowmax

@@ -28,16 +28,16 @@ EXACT_FP8_FEW_KEYS = 16
 EXACT_FP8_FEW_KEYS_TOL = 1e-1
 
 
-def run_cuda(wl: Workload, inp: Inputs, mode: int, device="cuda:0", tau=None):
+def run_cuda(wl: Workload, inp: Inputs, mode: int, device="cuda:0", tau=None, pot_tail=None):
     q, k, v = (t.to(device) for t in (inp.q, inp.k, inp.v))
     o, lse = binding.attn_fwd(q, k, v, causal=wl.causal, softmax_scale=wl.softmax_scale, weight_mode=mode,
                               q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale,
-                              rescale_tau=tau)
+                              rescale_tau=tau, pot_tail=pot_tail)
     torch.cuda.synchronize()
     return o, lse
 
 
-def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None, model_p_storage=False):
+def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None, model_p_storage=False, pot_tail=None):
     dt = {"bf16": orc.IN_BF16, "fp16": orc.IN_FP16, "fp8_e4m3": orc.IN_FP8_E4M3}[wl.in_dtype]
     sch = binding.get_schedule(wl.D, dt, mode, wl.causal)
     if mode == binding.W_EXACT_POLY:
@@ -45,6 +45,9 @@ def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None, model_
     assert sch["rescale_tau"] == 0.0
     if tau is not None:
         sch["rescale_tau"] = tau
+    drop_tail = False
+    if pot_tail is not None:
+        sch["pot_kmax"], drop_tail = int(pot_tail[0]), bool(pot_tail[1])
     tile = 0 if mode == orc.W_EXACT else sch["tile_n"]   # exact mode: the whole-row definition
     p_kw = {}
     if model_p_storage and sch["p_format"] == binding.P_E4M3:
@@ -53,13 +56,13 @@ def run_oracle(wl: Workload, inp: Inputs, mode: int, rows=None, tau=None, model_
         p_kw = {"p_round": orc.P_E4M3, "p_off": sch["p_offset_log2"]}
     return orc.attn(storage_bits(inp.q), storage_bits(inp.k), storage_bits(inp.v), in_dtype=dt,
                     causal=wl.causal, softmax_scale=wl.softmax_scale, mode=mode, tile_n=tile,
-                    kv_order=sch["kv_order"], tau=sch["rescale_tau"], kmax=sch["pot_kmax"],
+                    kv_order=sch["kv_order"], tau=sch["rescale_tau"], kmax=sch["pot_kmax"], drop_tail=drop_tail,
                     q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale,
                     tie_eps=TIE_EPS if mode != orc.W_EXACT else 0.0, rows=rows, **p_kw)
 
 
 def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, device="cuda:0",
-            allow_output_rounding: bool = False, tau=None, model_p_storage: bool = False):
+            allow_output_rounding: bool = False, tau=None, model_p_storage: bool = False, pot_tail=None):
     """Returns a dict of error statistics; `ok` says whether every gate holds.
 
     `model_p_storage`: where the kernel stores P in e4m3 (exact mode, and the eighth-octave family
@@ -71,8 +74,8 @@ def compare(wl: Workload, mode: int, inp: Inputs | None = None, rows=None, devic
     is stored in bf16, and for outputs of magnitude 2 and above that rounding alone is 0.008 and
     more.  The standard workloads (N(0,1) values, averaged) do not need it."""
     inp = inp or make_inputs(wl)
-    o, lse = run_cuda(wl, inp, mode, device, tau)
-    ref = run_oracle(wl, inp, mode, rows, tau, model_p_storage)
+    o, lse = run_cuda(wl, inp, mode, device, tau, pot_tail)
+    ref = run_oracle(wl, inp, mode, rows, tau, model_p_storage, pot_tail)
     o = o.float().cpu().numpy().transpose(0, 2, 1, 3).astype(np.float64)   # (B,Hq,Sq,D)
     lse = lse.cpu().numpy().astype(np.float64)
     if rows is not None:

@@ -61,3 +61,67 @@ def test_in_place_and_empty():
     assert x.cpu().tolist() == [0.375, 1.0]
     e = torch.empty(0, device="cuda")
     assert binding.weight_map(e, orc.W_H15).numel() == 0
+
+
+@pytest.mark.parametrize("drop", [False, True])
+@pytest.mark.parametrize("kmax", [1, 8, 12, 20, 48, 125])
+def test_pot_tail_map_is_bit_exact_on_the_sweep(kmax, drop):
+    for x in (inputs.weight_map_sweep(), inputs.paper_bit_test_set()):
+        x = x[x <= 0.5]
+        got = binding.weight_map_pot(torch.from_numpy(x).cuda(), kmax, drop).cpu().numpy()
+        want = orc.weight_map(x, orc.W_POT, kmax=kmax, drop_tail=drop).astype(np.float32)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def _chunks_of(x, pred):
+    """Offsets arranged so that chunks of 32 are uniform in `pred` (the fused loop picks its variant per chunk)."""
+    a, b = x[pred], x[~pred]
+    pad = (-len(a)) % 32
+    return np.concatenate([a, np.zeros(pad, np.float32), b]).astype(np.float32)
+
+
+# storage type -> (lowest offset whose weight P still holds exactly, per mode)
+_P_FLOOR = {
+    binding.IN_BF16: {orc.W_H15: -126.0, orc.W_H15K2: -126.0, orc.W_H15K3: -126.0, orc.W_POT: -126.0},
+    binding.IN_FP16: {orc.W_H15: -23.0, orc.W_POT: -24.0},     # fp16 subnormals: 1.5 * 2^k needs k >= -23
+    binding.IN_FP8_E4M3: {orc.W_H15: -29.0, orc.W_H15K2: -29.0, orc.W_H15K3: -14.0, orc.W_POT: -29.0},
+}
+
+
+@pytest.mark.parametrize("in_dtype", [binding.IN_BF16, binding.IN_FP16, binding.IN_FP8_E4M3])
+@pytest.mark.parametrize("mode", [orc.W_H15, orc.W_H15K2, orc.W_H15K3, orc.W_POT])
+def test_fused_loop_instantiations_are_bit_exact_where_p_holds_the_weight(mode, in_dtype):
+    # the instantiations attn_fwd runs (h15 family without the per-score clamp, P offset folded into the weight,
+    # pot on the negated offset), read back from the packed P words
+    if mode not in _P_FLOOR[in_dtype]:
+        pytest.skip("not built for this storage type")
+    floor = _P_FLOOR[in_dtype][mode]
+    kmax = {binding.IN_BF16: 20, binding.IN_FP16: 20, binding.IN_FP8_E4M3: 20}[in_dtype]
+    for x in (inputs.weight_map_sweep(), inputs.paper_bit_test_set()):
+        x = x[np.isfinite(x) & (x <= 0.0)]
+        x = _chunks_of(x, x >= -125.0)                    # chunks entirely above -125 take the unclamped variant
+        got = binding.weight_map_fused(torch.from_numpy(x).cuda(), mode, in_dtype, kmax).cpu().numpy()
+        want = orc.weight_map(x, mode, kmax=kmax).astype(np.float32)
+        held = x >= floor
+        assert np.array_equal(got[held].view(np.uint32), want[held].view(np.uint32))
+        # below that P rounds in its subnormal range and then underflows to zero: never more than one binade off
+        assert np.all(got[~held] >= 0) and np.all(got[~held] <= want[~held] * 2.0 + 2.0 ** -120)
+
+
+@pytest.mark.parametrize("in_dtype,kmax", [(binding.IN_BF16, 8), (binding.IN_BF16, 48), (binding.IN_FP8_E4M3, 12), (binding.IN_FP8_E4M3, 29),
+                                           (binding.IN_FP16, 12)])
+@pytest.mark.parametrize("drop", [False, True])
+def test_fused_loop_pot_tail(in_dtype, kmax, drop):
+    x = inputs.weight_map_sweep()
+    x = x[np.isfinite(x) & (x <= 0.0)]
+    got = binding.weight_map_fused(torch.from_numpy(x).cuda(), orc.W_POT, in_dtype, kmax, drop).cpu().numpy()
+    want = orc.weight_map(x, orc.W_POT, kmax=kmax, drop_tail=drop).astype(np.float32)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("in_dtype,rel", [(binding.IN_BF16, 2.0 ** -8), (binding.IN_FP16, 2.0 ** -11), (binding.IN_FP8_E4M3, 2.0 ** -4)])
+def test_fused_loop_exact_mode_is_the_exponential_rounded_to_the_format_of_p(in_dtype, rel):
+    x = np.linspace(-7.5, 0.0, 4096, dtype=np.float32)
+    got = binding.weight_map_fused(torch.from_numpy(x).cuda(), orc.W_EXACT, in_dtype).cpu().numpy().astype(np.float64)
+    want = orc.weight_map(x, orc.W_EXACT)
+    assert np.max(np.abs(got / want - 1.0)) <= rel * 1.01
