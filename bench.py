@@ -5,10 +5,17 @@
 
 A step is one attention forward in h15 mode over one synthetic batch of the headline workload
 (causal, 8192 keys, fp8 e4m3 inputs, B=2, 16 heads, D=128).  The same workload is also timed in
-exact mode, and its non-causal twin in both modes, for the H15-over-exact speed-up.  Inputs are
+exact mode, and its non-causal twin in both modes, for the H15-over-exact speed-up, with the paper's
+window protocol (Sec. 5.3, App. B "Measurement protocol and environment").  A matrix of further
+workloads (bf16, fp16, head dimension 64, grouped heads, 1K to 32K keys, Rowmax-PoT, the partly
+emulated exact control) follows with a lighter protocol; `--matrix none` skips it.  Inputs are
 resident in HBM for `value`; the `e2e` figure repeats the step from pinned host buffers with the
 copies inside the timed region.  With N > 1 (one process per GPU under torchrun) every rank runs an
 independent replica of the workload: the operator has no exchange step.
+
+    python bench.py --workload NAME --modes exact,h15 --launches 2
+
+runs one workload of the matrix a few times and prints its device time (for profilers).
 """
 from __future__ import annotations
 
@@ -36,7 +43,32 @@ METRIC = "attn_fwd_tflops_h15_causal_8k_fp8"
 # dram__bytes_read.sum + dram__bytes_write.sum of one h15 launch on the headline workload, from the ncu
 # capture summarised in profiles/attn_fwd_ws_causal_8k_fp8.txt (algorithmic: 101 MB in + 68 MB out)
 NCU_DRAM_BYTES_PER_LAUNCH = 171.8e6 + 32.6e6
-MODE_IDS = {"exact": 0, "pot": 1, "h15": 2}
+MODE_IDS = {"exact": 0, "pot": 1, "h15": 2, "h15k2": 3, "h15k3": 4, "exact_poly": 5}
+N_SMS = 148                   # B200
+MUFU_PER_CLK_PER_SM = 16      # ex2 results per clock per SM (Sec. 1)
+
+
+def matrix_workloads():
+    """(name, workload, modes): the timing matrix beside the headline.  Shapes follow the paper's B200 timing
+    tables (App. B: batch 1, 16 heads, D = 128, 1K to 32K keys; grouped heads 32/8; FP16; non-causal) and the
+    five configurations of the baseline description."""
+    paper = lambda name, S, causal, dt, D=128, seed=20: Workload(name, 1, 16, 16, S, S, D, causal, dt, seed)  # noqa: E731
+    out = [
+        ("causal_8k_bf16", paper("causal_8k_bf16", 8192, True, "bf16"), ("exact", "h15")),
+        ("noncausal_8k_bf16", paper("noncausal_8k_bf16", 8192, False, "bf16"), ("exact", "h15")),
+        ("causal_8k_fp16", paper("causal_8k_fp16", 8192, True, "fp16"), ("exact", "h15")),
+        ("gqa_causal_2k_bf16", WORKLOADS[1], ("exact", "h15")),
+        ("causal_16k_gqa_bf16", WORKLOADS[4], ("exact", "pot", "h15")),
+        ("causal_16k_gqa_fp8", WORKLOADS[4].with_(name="causal_16k_gqa_fp8", in_dtype="fp8_e4m3"), ("exact", "pot", "h15")),
+        ("causal_8k_bf16_d64", paper("causal_8k_bf16_d64", 8192, True, "bf16", D=64), ("exact", "h15")),
+        ("causal_8k_fp8_d64", paper("causal_8k_fp8_d64", 8192, True, "fp8_e4m3", D=64), ("exact", "h15")),
+    ]
+    for S in (1024, 2048, 4096, 8192, 16384, 32768):
+        nm = f"causal_{S // 1024}k_fp8_b1"
+        out.append((nm, paper(nm, S, True, "fp8_e4m3"), ("exact", "h15")))
+    out.append(("causal_8k_fp8_family", WORKLOADS[2].with_(name="causal_8k_fp8_family", B=1),
+                ("exact", "exact_poly", "pot", "h15", "h15k2", "h15k3")))
+    return out
 
 
 # ------------------------------------------------------------------------------------------------
@@ -242,25 +274,65 @@ class DeviceRun:
         return e0.elapsed_time(e1) / steps
 
 
-def speedup_rounds(run: DeviceRun, steps: int, device, rounds: int = 3):
-    """H15-over-exact speed-up as the paper measures it (Sec. 5.3): windows of back-to-back calls
-    between two CUDA events, the two modes in alternating order round by round (exact h15 / h15 exact /
-    exact h15), speed-up from the medians of each mode's pooled windows; the spread over rounds is
-    reported, not a confidence interval."""
-    windows = {"exact": [], "h15": []}
+def timed_windows(run: DeviceRun, modes, index: int, device, warmup: int, windows: int, calls: int, rounds: int):
+    """The paper's timing protocol (Sec. 5.3; App. B "Measurement protocol and environment"): `warmup` calls per
+    mode, then windows of `calls` back-to-back forwards between two CUDA events, `windows` per mode per round,
+    the modes in alternating order round by round (forward, reversed, forward, ...); per mode the median of its
+    pooled windows.  The SM clock is sampled while each mode's windows run."""
+    for name in modes:
+        for _ in range(warmup):
+            run.step(MODE_IDS[name])
+    torch.cuda.synchronize()
+    ms = {m: [] for m in modes}
+    mhz = {m: [] for m in modes}
     per_round = []
     for r in range(rounds):
-        order = ("exact", "h15") if r % 2 == 0 else ("h15", "exact")
+        order = list(modes) if r % 2 == 0 else list(reversed(modes))
         got = {}
         for name in order:
-            ms = max_over_ranks(run.time_steps(MODE_IDS[name], steps, 3), device)
-            windows[name].append(ms)
-            got[name] = ms
-        per_round.append(100.0 * (got["exact"] / got["h15"] - 1.0))
-    med = {k: statistics.median(v) for k, v in windows.items()}
-    return {"exact_ms": med["exact"], "h15_ms": med["h15"],
-            "h15_speedup_pct": 100.0 * (med["exact"] / med["h15"] - 1.0),
-            "speedup_pct_per_round": per_round, "windows_per_mode": rounds, "calls_per_window": steps}
+            with ClockSampler(index) as smp:
+                ws = [max_over_ranks(run.time_steps(MODE_IDS[name], calls, 0), device) for _ in range(windows)]
+            ms[name] += ws
+            got[name] = statistics.median(ws)
+            mhz[name] += [x[0] for x in smp.samples]
+        per_round.append(got)
+    out = {"protocol": {"warmup_calls": warmup, "windows_per_mode_per_round": windows, "calls_per_window": calls,
+                        "rounds": rounds, "order": "alternating"}, "modes": {}}
+    for name in modes:
+        med = statistics.median(ms[name])
+        clk = statistics.median(mhz[name]) if mhz[name] else None
+        out["modes"][name] = {"ms": med, "tflops": run.wl.flops / med / 1e9, "sm_mhz_median": clk,
+                              "ms_x_mhz": med * clk if clk else None,
+                              "ms_min": min(ms[name]), "ms_max": max(ms[name])}
+    if "exact" in modes:
+        for name in modes:
+            if name != "exact":
+                out["modes"][name]["speedup_over_exact_pct"] = 100.0 * (out["modes"]["exact"]["ms"] / out["modes"][name]["ms"] - 1.0)
+                out["modes"][name]["speedup_pct_per_round"] = [100.0 * (g["exact"] / g[name] - 1.0) for g in per_round]
+    return out
+
+
+def roofline_entries(res, wl: Workload, peaks):
+    """Fractions of the roofline per mode: the tensor bound against the measured cuBLAS bf16 rates (burst and
+    sustained; fp8 taken as twice bf16, the nominal ratio), and for the exact-like modes also the bound of the
+    special-function unit, one ex2 per visible score at 16 per clock per SM at the sampled SM clock; the
+    roofline of such a mode is the lower of the two."""
+    ratio = 2.0 if wl.in_dtype == "fp8_e4m3" else 1.0
+    scores = wl.flops / (4.0 * wl.D)                       # visible (query, key) pairs, by the same convention
+    for name, m in res["modes"].items():
+        tf = m["tflops"]
+        m["frac_tensor_burst"] = tf / (ratio * peaks["bf16_tflops"])
+        if peaks.get("bf16_tflops_sustained"):
+            m["frac_tensor_sustained"] = tf / (ratio * peaks["bf16_tflops_sustained"])
+        if name in ("exact", "exact_poly") and m.get("sm_mhz_median"):
+            share = 0.75 if name == "exact_poly" else 1.0   # a quarter of the scores bypasses the unit
+            bound_ms = 1e3 * share * scores / (MUFU_PER_CLK_PER_SM * N_SMS * m["sm_mhz_median"] * 1e6)
+            m["mufu_bound_ms"] = bound_ms
+            m["frac_mufu"] = bound_ms / m["ms"]
+            m["roofline_frac"] = max(m["frac_tensor_burst"], m["frac_mufu"])   # the lower bound in TFLOP/s = the larger fraction
+        else:
+            m["roofline_frac"] = m["frac_tensor_burst"]
+    return res
 
 
 def energy_leg(run: DeviceRun, index: int, seconds: float):
@@ -348,21 +420,21 @@ def run_ours(args):
     wl = HEADLINE
     inp = make_inputs(wl)
     run = DeviceRun(wl, inp, device)
-    twin_inp = make_inputs(TWIN)
-    twin = DeviceRun(TWIN, twin_inp, device)
     binding.device_status_reset()
+    peaks = measured_peaks()
 
     # headline: K steps of the h15 forward, clocks sampled during the region
     with ClockSampler(local_rank) as clk:
         n0 = binding.launch_count()
         ms_h15 = max_over_ranks(run.time_steps(MODE_IDS["h15"], args.steps, args.warmup), device)
         launches = binding.launch_count() - n0 - args.warmup
-        # exact mode of the same kernel and the non-causal twin, in alternating rounds
-        for _ in range(args.warmup):
-            run.step(MODE_IDS["exact"]); twin.step(MODE_IDS["exact"]); twin.step(MODE_IDS["h15"])
-        sp = speedup_rounds(run, args.steps, device)
-        sp_nc = speedup_rounds(twin, args.steps, device)
     clocks = clk.summary()
+    # exact mode of the same kernel and the non-causal twin: the paper's window protocol, independent of --steps
+    full = dict(warmup=50, windows=7, calls=100, rounds=3)
+    sp = roofline_entries(timed_windows(run, ("exact", "h15"), local_rank, device, **full), wl, peaks)
+    twin = DeviceRun(TWIN, make_inputs(TWIN), device)
+    sp_nc = roofline_entries(timed_windows(twin, ("exact", "h15"), local_rank, device, **full), TWIN, peaks)
+    del twin
     energy = energy_leg(run, local_rank, args.energy_seconds) if (world == 1 and args.energy_seconds > 0) else None
     ms_e2e, h2d, d2h = e2e_leg(run, max(3, args.steps // 4), args.warmup)
     ms_e2e = max_over_ranks(ms_e2e, device)
@@ -370,8 +442,24 @@ def run_ours(args):
     if status != 0:
         raise SystemExit(f"device-side wait expired during the bench (status {status:#x}); numbers invalid")
 
+    # the rest of the timing matrix (lighter protocol: a few seconds per entry)
+    matrix = {}
+    if args.matrix != "none":
+        light = dict(warmup=20, windows=3, calls=30, rounds=3)
+        for name, mwl, modes in matrix_workloads():
+            if args.matrix not in ("all", name):
+                continue
+            mrun = DeviceRun(mwl, make_inputs(mwl), device)
+            entry = roofline_entries(timed_windows(mrun, modes, local_rank, device, **light), mwl, peaks)
+            entry["config"] = {k: v for k, v in workload_config(mwl).items() if k not in ("weight_mode", "l2")}
+            matrix[name] = entry
+            del mrun
+            torch.cuda.empty_cache()
+        status = binding.device_status()
+        if status != 0:
+            raise SystemExit(f"device-side wait expired during the matrix (status {status:#x}); numbers invalid")
+
     tf = lambda w, ms: world * w.flops / ms / 1e9   # noqa: E731  (TFLOP/s, whole job)
-    peaks = measured_peaks()
     fp8_peak = 2.0 * peaks["bf16_tflops"]   # dense fp8 : bf16 nominal ratio is 2
     per_gpu = wl.flops / ms_h15 / 1e9
     line = {
@@ -387,13 +475,14 @@ def run_ours(args):
                      "peak_source": f"2 x {peaks['source']} cuBLAS bf16 burst ({peaks['bf16_tflops']} TFLOP/s); "
                                     "fp8 peak taken as twice the bf16 one (nominal ratio)",
                      "frac_of_nominal_fp8_4500": per_gpu / 4500.0},
-        "modes": {
-            "causal_8k_fp8": dict(sp, h15_tflops=tf(wl, sp["h15_ms"]), exact_tflops=tf(wl, sp["exact_ms"])),
-            "noncausal_8k_fp8": dict(sp_nc, h15_tflops=tf(TWIN, sp_nc["h15_ms"]), exact_tflops=tf(TWIN, sp_nc["exact_ms"])),
-        },
+        "modes": dict({"causal_8k_fp8": sp, "noncausal_8k_fp8": sp_nc}, **matrix),
     }
     if energy is not None:
         line["energy"] = energy
+        # the same step inside a loop of several seconds (power cap active): the sustained end of the headline
+        line["value_sustained"] = world * wl.flops / energy["h15"]["ms_per_forward"] / 1e9
+        line["roofline"]["frac_sustained"] = (wl.flops / energy["h15"]["ms_per_forward"] / 1e9) / (
+            2.0 * (peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]))
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg(wl, inp)
@@ -401,6 +490,28 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def run_workload(args):
+    """--workload NAME: a few launches of one workload per mode, device time from CUDA events (for profilers)."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention forward has no CPU path")
+    from paper_2609_33586_b200 import binding
+    table = {w.name: w for w in WORKLOADS}
+    table.update({n: w for n, w, _ in matrix_workloads()})
+    if args.workload not in table:
+        raise SystemExit(f"unknown workload {args.workload}; one of {sorted(table)}")
+    wl = table[args.workload]
+    if args.batch:
+        wl = wl.with_(B=args.batch)
+    run = DeviceRun(wl, make_inputs(wl), torch.device("cuda", 0))
+    binding.device_status_reset()
+    for name in args.modes.split(","):
+        ms = run.time_steps(MODE_IDS[name], args.launches, max(1, args.warmup_launches))
+        print(f"{wl.name} B={wl.B} {name}: {ms * 1e3:.1f} us per launch, {wl.flops / ms / 1e9:.1f} TFLOP/s")
+    status = binding.device_status()
+    if status != 0:
+        raise SystemExit(f"device-side wait expired (status {status:#x})")
 
 
 def main():
@@ -412,10 +523,18 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
     ap.add_argument("--energy-seconds", type=float, default=4.0,
                     help="length of the energy loop per mode at N=1 (0 = skip)")
+    ap.add_argument("--matrix", default="all", help="'all', 'none' or the name of one entry of the timing matrix")
+    ap.add_argument("--workload", default=None, help="profiling helper: run only this workload (see --modes, --launches)")
+    ap.add_argument("--batch", type=int, default=0, help="with --workload: override the batch size")
+    ap.add_argument("--modes", default="exact,h15", help="with --workload: weight modes to run")
+    ap.add_argument("--launches", type=int, default=2, help="with --workload: timed launches per mode")
+    ap.add_argument("--warmup-launches", type=int, default=1, help="with --workload: untimed launches per mode")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.workload is not None:
+        run_workload(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -137,14 +137,23 @@ int attn_weight_map_pot(const float* x, float* w, size_t n, int pot_kmax, int dr
 /*
  * attn_weight_map_fused — the weights as the hot loop of attn_fwd produces them and stores them in P for inputs of
  * storage type in_dtype (Eq. m-exact / Eq. rowmax-pot / Eq. h15 again, but through the instantiations the fused
- * kernel runs, which attn_weight_map does not reach: the h15 family without the per-score clamp wherever 32
- * consecutive offsets all lie above -125 octaves, with the clamp elsewhere; weights scaled by the P offset;
- * Rowmax-PoT evaluated on the negated offset, with the tail given here).  The n offsets are taken 32 at a time as
- * one chunk of a score row; the packed P words are decoded again and divided by the P scale.  For the lattice
- * maps the result equals attn_weight_map bit for bit wherever P can hold the weight: everywhere for bf16 P, down
- * to 2^-23 for fp16 P (powers of two: 2^-24), down to 2^-29 for e5m2 P (pot, h15, h15k2 on fp8 inputs) and down to 2^-14
- * for e4m3 P (h15k3 on fp8 inputs); below that P underflows towards zero.  exact-like modes are rounded to the
- * format of P.  pot_kmax / drop_tail matter in ATTN_W_POT mode only (limits as for attn_fwd_pot).
+ * kernel runs, which attn_weight_map does not reach).  The n offsets are taken 32 at a time as one chunk of a
+ * score row (score = offset, anchor 0, scale 1); the packed P words are decoded again and divided by the P scale.
+ *   fp8 inputs, h15 family: the packed form without the per-score clamp wherever the 32 offsets all lie above -125
+ *     octaves, with the clamp elsewhere; weights scaled by the P offset.  Equal to attn_weight_map bit for bit
+ *     wherever P holds the weight: down to 2^-29 (e5m2 P: h15, h15k2) or 2^-14 (e4m3 P: h15k3).
+ *   16-bit inputs, h15 family: the saturating form (scale, anchor shift and lower clamp in one saturating
+ *     multiply-add on the distance below the anchor, then one multiply-add that rounds).  The rounded integer is
+ *     that of Eq. h15 except possibly for offsets within 2^-20 (relative) of a rounding tie, where the fp32
+ *     rounding of the scaled distance decides; everywhere else equal to attn_weight_map bit for bit (bf16 P
+ *     holds every weight; fp16 P down to 2^-23).
+ *   Rowmax-PoT: the offset rounded to the nearest integer by the same add as h15 (ties to even, where Eq. rowmax-pot
+ *     sends ties down: the two differ only at an exact tie x = -(d + 1/2), d odd, where the fused loop gives the
+ *     larger neighbour; the boundary of a dropped tail is kept as defined), with the tail given here; bit for bit
+ *     elsewhere, wherever P holds the weight (fp16 P: 2^-24, e5m2 P: 2^-29).
+ *   exact-like modes: 2^x rounded to the format of P.
+ * Below the range of P the stored weight rounds in the subnormal range of the format and then underflows to zero.
+ * pot_kmax / drop_tail matter in ATTN_W_POT mode only (limits as for attn_fwd_pot).
  */
 int attn_weight_map_fused(const float* x, float* w, size_t n, int weight_mode, int in_dtype,
                           int pot_kmax, int drop_tail, void* stream);

@@ -14,8 +14,8 @@ cudaError_t launch_attn_fwd(int D, int in_type, int mode, const CUtensorMap& tq,
                             const CUtensorMap& tv, const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cudaStream_t stream);
 cudaError_t launch_weight_map_pot(const float* x, float* w, size_t n, int kmax, int drop, cudaStream_t stream);
-cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_cap,
-                                    float pot_drop_y, cudaStream_t stream);
+cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_neg_cap,
+                                    float pot_drop_x, cudaStream_t stream);
 cudaError_t status_word_address(int** out);
 }  // namespace rowmax
 
@@ -166,8 +166,8 @@ int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, i
     p.v_descale = fp8 ? v_descale : 1.0f;
     p.two22 = 1u << 22;
     p.tau = rescale_tau;
-    p.pot_cap = static_cast<float>(pot_kmax) + (drop ? 1.25f : 0.25f);
-    p.pot_drop_y = drop ? static_cast<float>(pot_kmax) + 0.5f : INFINITY;
+    p.pot_neg_cap = -static_cast<float>(drop ? pot_kmax + 1 : pot_kmax);
+    p.pot_drop_x = -(static_cast<float>(pot_kmax) + 0.5f);
 
 #ifdef ROWMAX_TRACE
     p.trace = g_trace;
@@ -184,7 +184,8 @@ int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, i
 
     static_assert(ATTN_IN_BF16 == rowmax::kInBF16 && ATTN_IN_FP8_E4M3 == rowmax::kInFP8 && ATTN_IN_FP16 == rowmax::kInFP16,
                   "the kernel's storage-type codes are those of the C interface");
-    cudaError_t e = rowmax::launch_attn_fwd(D, in_dtype, weight_mode, tq, tk, tv, p, static_cast<cudaStream_t>(stream));
+    const int kernel_mode = (weight_mode == ATTN_W_POT && drop) ? rowmax::kPotDrop : weight_mode;
+    cudaError_t e = rowmax::launch_attn_fwd(D, in_dtype, kernel_mode, tq, tk, tv, p, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(e);
         return e == cudaErrorInvalidValue ? ATTN_ERR_UNSUPPORTED : ATTN_ERR_CUDA;
@@ -253,9 +254,9 @@ int attn_weight_map_fused(const float* x, float* w, size_t n, int weight_mode, i
     const int kmax_hi = in_dtype == ATTN_IN_FP8_E4M3 ? ATTN_POT_KMAX_FP8 : (in_dtype == ATTN_IN_FP16 ? ATTN_POT_KMAX_FP16 : ATTN_POT_KMAX_BF16);
     if (weight_mode == ATTN_W_POT && (pot_kmax < 1 || pot_kmax > kmax_hi)) return ATTN_ERR_BAD_VALUE;
     const bool drop = drop_tail != 0;
-    cudaError_t e = rowmax::launch_weight_map_fused(x, w, n, weight_mode, in_dtype, static_cast<float>(pot_kmax) + (drop ? 1.25f : 0.25f),
-                                                    drop ? static_cast<float>(pot_kmax) + 0.5f : INFINITY,
-                                                    static_cast<cudaStream_t>(stream));
+    const int kernel_mode = (weight_mode == ATTN_W_POT && drop) ? rowmax::kPotDrop : weight_mode;
+    cudaError_t e = rowmax::launch_weight_map_fused(x, w, n, kernel_mode, in_dtype, -static_cast<float>(drop ? pot_kmax + 1 : pot_kmax),
+                                                    -(static_cast<float>(pot_kmax) + 0.5f), static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(e);
         return e == cudaErrorInvalidValue ? ATTN_ERR_UNSUPPORTED : ATTN_ERR_CUDA;

@@ -379,6 +379,13 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t tO = tmem_O(t) + lane_base;
         constexpr int kFam = h15_family_k(MODE);   // h15 family: the map takes the offset times 2^kFam
         const float c_eff = static_cast<float>(1 << kFam) * p.c;
+        // 16-bit inputs: the h15 family uses the saturating form of weights_chunk32 (no row-minimum pass, no
+        // clamped or masked variants) whenever the anchor is always current (offsets <= 0); the deferred rescale,
+        // where a score may lie above its anchor, keeps the form with explicit clamps.  fp8 inputs keep the
+        // packed form: there a bound on the key magnitude already removes the row-minimum pass, and the
+        // scalar multiply-adds of the saturating form cost more issue slots than they save (measured 4 to 6 %).
+        constexpr bool kLattice = kFam > 0 && !FP8;
+        const bool sat_form = kLattice && (IN != kInBF16 || !(p.tau > 0.0f));
         int tiles = 0;
         for (int round = 0;; ++round) {
             const int w = item_index(round, cta, n_ctas);
@@ -448,19 +455,31 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 RowScale rs;
                 float nmc = (is_exact_like(MODE) ? p_off : 0.0f) - m_use * c_eff;
                 float c_row = c_eff;
-                if constexpr (MODE == kPot) {   // pot works on y = -x = m*c - s*c
-                    nmc = -nmc;
-                    c_row = -c_eff;
-                }
                 rs.c = make_float2(c_row, c_row);
                 rs.nmc = make_float2(nmc, nmc);
                 rs.two22 = p.two22;
-                rs.pot_cap = p.pot_cap;
-                rs.pot_drop_y = p.pot_drop_y;
+                rs.pot_neg_cap = p.pot_neg_cap;
+                rs.pot_drop_x = p.pot_drop_x;
                 rs.clamp_lo = 0.f;
                 if constexpr (kFam > 0) rs.clamp_lo = masked_tile ? h15_clamp_zero<kFam>() : h15_clamp_floor<kFam>();
                 float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                if ((MODE == kPot || MODE == kExactPoly) && masked_tile) {
+                if (kLattice && sat_form) {
+                    // distance below the anchor as a fraction of the clamp distance R, which is also where a masked
+                    // score (-inf) ends up: 2^K * 126 (weight floor 2^-126, Eq. h15), in a tile with masked scores
+                    // 2^K * 127 (pattern of +0)
+                    constexpr float kR = 126.0f * (1 << kFam), kRm = 127.0f * (1 << kFam);
+                    const float big_r = masked_tile ? kRm : kR;
+                    const float inv_r = masked_tile ? 1.0f / kRm : 1.0f / kR;
+                    rs.su = -c_eff * inv_r;
+                    rs.ou = (m_use * c_eff) * inv_r;
+                    rs.sat_mul = -big_r;
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t pw[16];
+                        weights_chunk32<FP8, MODE, false, true, HALF, true>(s[cc], rs, 32, acc, pw);
+                        tmem_st16(tS + cc * 16, pw);
+                    }
+                } else if ((is_pot(MODE) || MODE == kExactPoly) && masked_tile) {
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t pw[16];
@@ -604,6 +623,7 @@ static cudaError_t dispatch_mode(int mode, const CUtensorMap& tq, const CUtensor
     switch (mode) {
         case kExact: return launch_ws<D, IN, kExact>(tq, tk, tv, p, stream);
         case kPot: return launch_ws<D, IN, kPot>(tq, tk, tv, p, stream);
+        case kPotDrop: return launch_ws<D, IN, kPotDrop>(tq, tk, tv, p, stream);
         case kH15: return launch_ws<D, IN, kH15>(tq, tk, tv, p, stream);
         default: break;
     }
@@ -672,12 +692,12 @@ cudaError_t launch_weight_map_pot(const float* x, float* w, size_t n, int kmax, 
 
 // The weights as the fused kernel's hot loop produces and stores them: every thread takes 32 consecutive offsets
 // as one chunk of a score row (score = offset, scale 1, anchor 0), runs weights_chunk32 with the template
-// arguments of the fused kernel for that storage type, including its choice between the unclamped and the
-// clamped h15 variant (here per chunk; in the fused kernel per warp and key tile), and decodes the packed P
-// words back to fp32, divided by the P scale.
+// arguments of the fused kernel for that storage type (fp8: its choice between the unclamped and the clamped h15
+// variant, here per chunk, in the fused kernel per warp and key tile; 16 bit: the saturating form), and decodes
+// the packed P words back to fp32, divided by the P scale.
 template <bool FP8, bool HALF, int MODE>
 __global__ void weight_map_fused_kernel(const float* __restrict__ x, float* __restrict__ w, size_t n, uint32_t two22,
-                                        float pot_cap, float pot_drop_y) {
+                                        float pot_neg_cap, float pot_drop_x) {
     constexpr int kFam = h15_family_k(MODE);
     constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
     const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
@@ -692,20 +712,29 @@ __global__ void weight_map_fused_kernel(const float* __restrict__ x, float* __re
             lowest = fminf(lowest, xi);
         }
         RowScale rs;
-        const float c_row = kFam > 0 ? static_cast<float>(1 << kFam) : (MODE == kPot ? -1.0f : 1.0f);
+        const float c_row = static_cast<float>(1 << kFam);
         const float nmc = is_exact_like(MODE) ? static_cast<float>(kOff) : 0.0f;
         rs.c = make_float2(c_row, c_row);
         rs.nmc = make_float2(nmc, nmc);
         rs.two22 = two22;
-        rs.pot_cap = pot_cap;
-        rs.pot_drop_y = pot_drop_y;
+        rs.pot_neg_cap = pot_neg_cap;
+        rs.pot_drop_x = pot_drop_x;
         rs.clamp_lo = 0.f;
         if constexpr (kFam > 0) rs.clamp_lo = h15_clamp_floor<kFam>();
         float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         uint32_t pw[16];
-        const bool clamp = kFam > 0 && !(lowest * (1 << kFam) >= -125.0f * (1 << kFam));
-        if (clamp) weights_chunk32<FP8, MODE, false, true, HALF>(s, rs, 32, acc, pw);
-        else weights_chunk32<FP8, MODE, false, false, HALF>(s, rs, 32, acc, pw);
+        if constexpr (kFam > 0 && !FP8) {
+            // 16-bit inputs: the saturating form, as in a key tile without masked scores
+            constexpr float kR = 126.0f * (1 << kFam);
+            rs.su = -static_cast<float>(1 << kFam) * (1.0f / kR);
+            rs.ou = 0.0f;
+            rs.sat_mul = -kR;
+            weights_chunk32<FP8, MODE, false, true, HALF, true>(s, rs, 32, acc, pw);
+        } else {
+            const bool clamp = kFam > 0 && !(lowest * (1 << kFam) >= -125.0f * (1 << kFam));
+            if (clamp) weights_chunk32<FP8, MODE, false, true, HALF>(s, rs, 32, acc, pw);
+            else weights_chunk32<FP8, MODE, false, false, HALF>(s, rs, 32, acc, pw);
+        }
         const float unscale = __uint_as_float(static_cast<uint32_t>(127 - kOff) << 23);   // 2^-kOff
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -731,21 +760,22 @@ __global__ void weight_map_fused_kernel(const float* __restrict__ x, float* __re
 }
 
 template <bool FP8, bool HALF>
-static cudaError_t launch_fused_map_mode(const float* x, float* w, size_t n, int mode, float pot_cap, float pot_drop_y,
+static cudaError_t launch_fused_map_mode(const float* x, float* w, size_t n, int mode, float pot_neg_cap, float pot_drop_x,
                                          cudaStream_t stream) {
     size_t blocks = ((n + 31) / 32 + 127) / 128;
     if (blocks > 148 * 8) blocks = 148 * 8;
     const unsigned g = static_cast<unsigned>(blocks);
     switch (mode) {
-        case kExact: weight_map_fused_kernel<FP8, HALF, kExact><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
-        case kPot: weight_map_fused_kernel<FP8, HALF, kPot><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
-        case kH15: weight_map_fused_kernel<FP8, HALF, kH15><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+        case kExact: weight_map_fused_kernel<FP8, HALF, kExact><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
+        case kPot: weight_map_fused_kernel<FP8, HALF, kPot><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
+        case kPotDrop: weight_map_fused_kernel<FP8, HALF, kPotDrop><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
+        case kH15: weight_map_fused_kernel<FP8, HALF, kH15><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
         default:
             if constexpr (!HALF) {
                 switch (mode) {
-                    case kH15K2: weight_map_fused_kernel<FP8, HALF, kH15K2><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
-                    case kH15K3: weight_map_fused_kernel<FP8, HALF, kH15K3><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
-                    case kExactPoly: weight_map_fused_kernel<FP8, HALF, kExactPoly><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_cap, pot_drop_y); break;
+                    case kH15K2: weight_map_fused_kernel<FP8, HALF, kH15K2><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
+                    case kH15K3: weight_map_fused_kernel<FP8, HALF, kH15K3><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
+                    case kExactPoly: weight_map_fused_kernel<FP8, HALF, kExactPoly><<<g, 128, 0, stream>>>(x, w, n, 1u << 22, pot_neg_cap, pot_drop_x); break;
                     default: return cudaErrorInvalidValue;
                 }
             } else {
@@ -755,12 +785,12 @@ static cudaError_t launch_fused_map_mode(const float* x, float* w, size_t n, int
     return cudaGetLastError();
 }
 
-cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_cap,
-                                    float pot_drop_y, cudaStream_t stream) {
+cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_neg_cap,
+                                    float pot_drop_x, cudaStream_t stream) {
     if (n == 0) return cudaSuccess;
-    if (in_type == kInFP8) return launch_fused_map_mode<true, false>(x, w, n, mode, pot_cap, pot_drop_y, stream);
-    if (in_type == kInFP16) return launch_fused_map_mode<false, true>(x, w, n, mode, pot_cap, pot_drop_y, stream);
-    return launch_fused_map_mode<false, false>(x, w, n, mode, pot_cap, pot_drop_y, stream);
+    if (in_type == kInFP8) return launch_fused_map_mode<true, false>(x, w, n, mode, pot_neg_cap, pot_drop_x, stream);
+    if (in_type == kInFP16) return launch_fused_map_mode<false, true>(x, w, n, mode, pot_neg_cap, pot_drop_x, stream);
+    return launch_fused_map_mode<false, false>(x, w, n, mode, pot_neg_cap, pot_drop_x, stream);
 }
 
 cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cudaStream_t stream) {

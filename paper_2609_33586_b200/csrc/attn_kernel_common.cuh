@@ -10,7 +10,10 @@ constexpr int kTileN = 128;  // keys per tile
 
 // storage type of q, k, v (the values of ATTN_IN_* in the C interface)
 enum InType : int { kInBF16 = 0, kInFP8 = 1, kInFP16 = 2 };
-enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4, kExactPoly = 5 };
+// kPotDrop is internal: Rowmax-PoT with a dropped tail (the C interface selects it through attn_fwd_pot), a
+// separate instance so that the clamped tail does not pay for the comparison that drops.
+enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4, kExactPoly = 5, kPotDrop = 6 };
+__host__ __device__ constexpr bool is_pot(int mode) { return mode == kPot || mode == kPotDrop; }
 // modes whose weight is 2^x itself (with the P offset folded into x)
 __host__ __device__ constexpr bool is_exact_like(int mode) { return mode == kExact || mode == kExactPoly; }
 // input-rounding exponent of the h15 family member: steps of 2^-k octaves (0: not a family member)
@@ -29,8 +32,8 @@ struct AttnParams {
     float tau;        // rescale threshold in octaves (0 = the anchor is always the running maximum)
     uint32_t two22;   // 1 << 22, kept in a register for the h15 integer multiply-add
     // Rowmax-PoT tail (Eq. rowmax-pot and the sentence after it): index cap K_max and what happens beyond it
-    float pot_cap;    // y = -x is capped at K_max + 1/4 (clamped tail) or K_max + 1 + 1/4 (dropped tail)
-    float pot_drop_y; // dropped tail: y at or above K_max + 1/2 weighs zero; +inf with a clamped tail
+    float pot_neg_cap;  // lower clamp of the offset: -K_max (clamped tail) or -(K_max + 1) (dropped tail)
+    float pot_drop_x;   // dropped tail: offsets below -(K_max + 1/2) weigh zero
     int* status;      // device-global sticky status word
 #ifdef ROWMAX_TRACE
     long long* trace;  // optional per-role cycle stamps of one CTA: [role 4][tile 64][slot 8]

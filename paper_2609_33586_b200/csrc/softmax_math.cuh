@@ -176,16 +176,34 @@ struct RowScale {
     float2 nmc;    // minus the scaled anchor (plus the P offset in exact mode), both lanes
     uint32_t two22;  // 1 << 22 held in a register (see imad)
     float clamp_lo;  // h15 family, clamped variant: lower bound of the scaled offset (see w_h15_doubled_pair)
-    float pot_cap;   // pot: cap of y = -x (K_max + 1/4, or K_max + 1 + 1/4 with a dropped tail)
-    float pot_drop_y;  // pot, dropped tail: y at or above this (K_max + 1/2) weighs zero; +inf: nothing is dropped
+    float pot_neg_cap;  // pot: lower clamp of the offset, -K_max (clamped tail) or -(K_max + 1) (dropped tail)
+    float pot_drop_x;   // pot, dropped tail: offsets at or below this (-(K_max + 1/2)) weigh zero
+    // saturating form (SAT, h15 family): u = sat(score * su + ou) is the distance below the anchor as a fraction
+    // of the clamp distance R = 2^K * 126 (2^K * 127 in a tile with masked scores); sat_mul = -R
+    float su, ou, sat_mul;
 };
+
+// fma with saturation to [0, 1] (NaN gives 0)
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 // Turns 32 consecutive scores of one row into weights.  Adds them (times 2^kOffLog2) into `acc`
 // (two independent packed accumulators, summed by the caller)
 // and writes the packed P words: 16 words of 2 bf16 (2 fp16 with HALFP), or 8 words of 4 fp8.  In a MASKED tile
 // columns >= limit are masked: their scores already hold -inf and their weights are forced to 0.
 // CLAMP = false (h15 only) may be used when every doubled offset of the chunk is known to be >= -252.
-template <bool FP8, int MODE, bool MASKED, bool CLAMP = true, bool HALFP = false>
+// SAT (h15 family, anchor always current): the scale, the shift by the anchor and the lower clamp are one
+// saturating multiply-add, u = sat((anchor - score) c' / R) in [0, 1], small and therefore accurate near the anchor;
+// the second multiply-add puts R u back and adds the rounding constant in one rounding: t = 2^23 + 2^22 - R u, the
+// integer n = -RNE(R u), clamped at -R.  No clamped or unclamped variants, no row minimum: a score further than R
+// below its anchor, and a masked score (-inf), saturate.  With R = 2^K * 126 the saturated weight is the floor
+// 2^-126 of Eq. h15; a key tile with masked scores uses R = 2^K * 127, whose saturated pattern is +0, so that a
+// masked score weighs exactly nothing.  The integer is that of Eq. h15 up to the fp32 rounding of u (relative
+// 2^-23 of the distance), i.e. it can differ only for offsets that close to a rounding tie.
+template <bool FP8, int MODE, bool MASKED, bool CLAMP = true, bool HALFP = false, bool SAT = false>
 __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const RowScale& rs, int limit,
                                                 float2 (&acc)[2], uint32_t* pw) {
     constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
@@ -193,9 +211,15 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const float2 sv = make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
-        float2 x = ffma2(sv, rs.c, rs.nmc);
+        float2 x = make_float2(0.f, 0.f);
+        if constexpr (!SAT) x = ffma2(sv, rs.c, rs.nmc);
         float2 w;
-        if constexpr (MODE == kExactPoly && !MASKED) {
+        if constexpr (SAT && h15_family_k(MODE) > 0) {
+            float2 t;
+            t.x = fmaf(fma_sat(sv.x, rs.su, rs.ou), rs.sat_mul, kH15Magic);
+            t.y = fmaf(fma_sat(sv.y, rs.su, rs.ou), rs.sat_mul, kH15Magic);
+            w = h15_weight_pair_from_t<kOff, h15_family_k(MODE)>(t, rs.two22);
+        } else if constexpr (MODE == kExactPoly && !MASKED) {
             // every fourth pair (25 % of the scores) takes the polynomial route, the rest the hardware ex2
             if (i % 4 == 3) {
                 w.x = w_exact_poly3(x.x);
@@ -212,11 +236,11 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             // integer n, ties to even), then (bits << (23 - K)) + bias builds the weight times 2^kOff.
             w = w_h15_doubled_pair<kOff, CLAMP, h15_family_k(MODE)>(x, rs.two22, rs.clamp_lo);
         } else {
-            // rs.c and rs.nmc carry the opposite sign in pot mode: x holds y = -(offset) >= 0
-            w.x = pot_weight_from_y<kOff>(x.x, rs.pot_cap);
-            w.y = pot_weight_from_y<kOff>(x.y, rs.pot_cap);
-            if (x.x >= rs.pot_drop_y) w.x = 0.f;
-            if (x.y >= rs.pot_drop_y) w.y = 0.f;
+            w = pot_weight_pair_rne<kOff>(x, rs.pot_neg_cap, rs.two22 << 1);
+            if constexpr (MODE == kPotDrop) {   // the index K_max + 1 stands for everything beyond K_max: weight zero
+                if (x.x <= rs.pot_drop_x) w.x = 0.f;
+                if (x.y <= rs.pot_drop_x) w.y = 0.f;
+            }
         }
         if constexpr (!is_exact_like(MODE) && MASKED) {
             if (2 * i >= limit) w.x = 0.f;

@@ -56,6 +56,17 @@ __device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_fro
 // inputs are at or above -126 * 2^K.  The clamp value is -126 * 2^K (Eq. h15: the weight floor 2^-126);
 // the fused kernel passes -127 * 2^K in a key tile that holds masked scores: that input gives the
 // bit pattern of +0 (times 2^kOff), so a masked score (-inf) weighs exactly nothing.
+// Two rounded patterns t = 2^23 + 2^22 + n (as floats) -> the two weights (1 + (n mod 2^K) / 2^K) 2^floor(n / 2^K)
+// times 2^kOff: (bits << (23 - K)) + bias, one lane by shift-add (ALU pipe), the other by the equivalent integer
+// multiply-add (FMA pipe).
+template <int kOff, int K>
+__device__ __forceinline__ float2 h15_weight_pair_from_t(float2 t, uint32_t two22) {
+    constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(kOff) << 23);
+    const uint32_t b0 = (__float_as_uint(t.x) << (23 - K)) + bias;
+    uint32_t b1;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22 >> (K - 1)), "r"(bias));
+    return make_float2(__uint_as_float(b0), __uint_as_float(b1));
+}
 template <int K>
 __device__ __forceinline__ constexpr float h15_clamp_floor() { return -126.0f * (1 << K); }
 template <int K>
@@ -74,11 +85,7 @@ __device__ __forceinline__ float2 w_h15_doubled_pair(float2 x2, uint32_t two22, 
         "mov.b64 {%0, %1}, rd;\n\t}"
         : "=f"(t.x), "=f"(t.y)
         : "f"(x2.x), "f"(x2.y), "f"(kH15Magic));
-    constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(kOff) << 23);
-    const uint32_t b0 = (__float_as_uint(t.x) << (23 - K)) + bias;
-    uint32_t b1;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two22 >> (K - 1)), "r"(bias));
-    return make_float2(__uint_as_float(b0), __uint_as_float(b1));
+    return h15_weight_pair_from_t<kOff, K>(t, two22);
 }
 
 // ---- Rowmax-PoT (Eq. rowmax-pot): d = min{K_max, floor(y + 1/2)}, y = -x, w = 2^-d.
@@ -103,8 +110,36 @@ __device__ __forceinline__ int pot_index(float x) { return pot_index_from_y(-x);
 // the t pattern without its lowest bit, shifted right by one: ((tbits & ~1) << 22) puts it at bit 23
 // (the bits of 2^22's own pattern fall off the top).
 template <int kOff>
+__device__ __forceinline__ float pot_weight_from_tbits(uint32_t tbits) {
+    return __uint_as_float((static_cast<uint32_t>(191 + kOff) << 23) - ((tbits & ~1u) << 22));
+}
+template <int kOff>
 __device__ __forceinline__ float pot_weight_from_y(float y, float cap = kPotCapDefault) {
-    return __uint_as_float((static_cast<uint32_t>(191 + kOff) << 23) - ((pot_tbits(y, cap) & ~1u) << 22));
+    return pot_weight_from_tbits<kOff>(pot_tbits(y, cap));
+}
+// Two at once, the form the fused kernel uses, on the offsets x themselves.  -floor(-x + 1/2) = ceil(x - 1/2) is x
+// rounded to the nearest integer with ties going DOWN; adding 2^23 + 2^22 rounds to nearest with ties to EVEN, the
+// same integer except at an exact tie (x = k + 1/2 with k odd).  Inside the fused kernel x is itself an fp32
+// rounding of the true offset, so an exact tie carries no information and this costs nothing; the stand-alone map
+// above keeps the definition.  Then the pattern of 2^(n + kOff) is (bits << 23) + bias, one lane by shift-add, the
+// other by the equivalent integer multiply-add (two23 must hold 1 << 23).  The lower clamp -cap (cap = K_max, or
+// K_max + 1 with a dropped tail, at most 125) keeps the index in range and makes min{K_max, .} implicit.
+template <int kOff>
+__device__ __forceinline__ float2 pot_weight_pair_rne(float2 x, float neg_cap, uint32_t two23) {
+    x.x = fmaxf(x.x, neg_cap);
+    x.y = fmaxf(x.y, neg_cap);
+    float2 t;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(t.x), "=f"(t.y)
+        : "f"(x.x), "f"(x.y), "f"(kH15Magic));
+    constexpr uint32_t bias = 0x3F800000u + (static_cast<uint32_t>(kOff) << 23);
+    const uint32_t b0 = (__float_as_uint(t.x) << 23) + bias;
+    uint32_t b1;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(b1) : "r"(__float_as_uint(t.y)), "r"(two23), "r"(bias));
+    return make_float2(__uint_as_float(b0), __uint_as_float(b1));
 }
 __device__ __forceinline__ float w_pot(float x) { return pot_weight_from_y<0>(-x); }
 // General tail: K_max as a run-time value, clamped (every key keeps 2^-K_max) or dropped (weight zero
