@@ -56,7 +56,7 @@ enum {
     ATTN_ERR_MISALIGNED = -4,       /* q, k, v or o not 16-byte aligned */
     ATTN_ERR_UNSUPPORTED_ARCH = -5, /* current device is not compute capability 10.x */
     ATTN_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed; see attn_last_cuda_error */
-    ATTN_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired; see attn_device_status */
+    ATTN_ERR_TIMEOUT = -7,          /* returned by attn_device_status: a bounded device-side wait has expired */
     ATTN_ERR_UNSUPPORTED = -8,      /* valid arguments, combination not built (e.g. a deferred rescale on fp8 inputs) */
     ATTN_ERR_BAD_VALUE = -9         /* softmax_scale or an fp8 descale not positive and finite; rescale_tau or K_max out of range */
 };
@@ -174,13 +174,27 @@ int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal,
                       int* pot_kmax, int* p_format, int* p_offset_log2);
 
 /*
- * attn_device_status — synchronises the current device and returns the sticky device-side status
- * word: 0, or a code telling which bounded wait expired (role << 8 | barrier id).  A non-zero
- * value means results of the affected launch are invalid.  attn_device_status_reset clears it.
- * (No counterpart in the paper: safety net for the mbarrier/TMEM pipeline.)
+ * Device-side waits and the status word.  (No counterpart in the paper: safety net of the mbarrier / TMEM pipeline.)
+ * Every wait inside the kernels is bounded (about one second).  A wait that runs out writes a code, role << 8 |
+ * barrier id, into one status word per device, and the kernel winds down: the roles leave their loops, copies and
+ * MMAs in flight are awaited with a bound, nothing more is stored, TMEM is released.  No trap, no hang.
+ * The word is STICKY: it stays set across launches until attn_device_status_reset.  While it is set, attn_fwd,
+ * attn_fwd_tau and attn_fwd_pot still return ATTN_OK (they are asynchronous and do not read the word), but their
+ * kernels return at once WITHOUT writing o or lse.  So: after a batch of launches call attn_device_status; on
+ * ATTN_ERR_TIMEOUT treat every output since the last clean check as invalid, reset, and launch again.
+ *   attn_device_status        synchronises the current device; ATTN_OK, ATTN_ERR_TIMEOUT (the word is set), or
+ *                             ATTN_ERR_CUDA
+ *   attn_device_status_code   same, but returns the word itself (0, or role << 8 | barrier id of the first wait
+ *                             that ran out) or a negative ATTN_ERR_*
+ *   attn_device_status_reset  synchronises and clears the word
+ *   attn_selftest_wait        launches one warp that waits, for at most limit_cycles SM clocks (1 .. 2e9), on a
+ *                             barrier that nothing arrives on: the wait runs out, the word is set (role 7, barrier
+ *                             0x7f) and the kernel returns.  For tests of the path above; clear the word afterwards.
  */
 int attn_device_status(void);
+int attn_device_status_code(void);
 int attn_device_status_reset(void);
+int attn_selftest_wait(long long limit_cycles, void* stream);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 unsigned long long attn_launch_count(void);

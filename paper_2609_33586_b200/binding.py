@@ -21,7 +21,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libattn_b200.so"
 _lib = None
 
 EXPORTS = ("attn_fwd", "attn_fwd_tau", "attn_fwd_pot", "attn_weight_map", "attn_weight_map_pot", "attn_weight_map_fused", "attn_get_schedule", "attn_device_status",
-           "attn_device_status_reset", "attn_launch_count", "attn_status_string",
+           "attn_device_status_code", "attn_selftest_wait", "attn_device_status_reset", "attn_launch_count", "attn_status_string",
            "attn_last_cuda_error", "attn_version")
 
 
@@ -55,6 +55,9 @@ def lib() -> ctypes.CDLL:
         L.attn_get_schedule.restype = i
         L.attn_get_schedule.argtypes = [i, i, i, i] + [vp] * 7
         L.attn_device_status.restype = i
+        L.attn_device_status_code.restype = i
+        L.attn_selftest_wait.restype = i
+        L.attn_selftest_wait.argtypes = [ctypes.c_longlong, vp]
         L.attn_device_status_reset.restype = i
         L.attn_launch_count.restype = ctypes.c_ulonglong
         L.attn_status_string.restype = ctypes.c_char_p
@@ -79,6 +82,18 @@ def launch_count() -> int:
 
 def device_status() -> int:
     return int(lib().attn_device_status())
+
+
+def device_status_code() -> int:
+    """The raw status word: 0, or role << 8 | barrier id of the first wait that ran out."""
+    return int(lib().attn_device_status_code())
+
+
+def selftest_wait(limit_cycles: int, stream=None) -> None:
+    """Launches the one-warp kernel whose bounded wait runs out (sets the sticky status word)."""
+    rc = lib().attn_selftest_wait(int(limit_cycles), _stream_ptr(stream))
+    if rc != 0:
+        raise AttnError(rc, "attn_selftest_wait")
 
 
 def device_status_reset() -> None:

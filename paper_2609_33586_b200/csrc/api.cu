@@ -17,6 +17,7 @@ cudaError_t launch_weight_map_pot(const float* x, float* w, size_t n, int kmax, 
 cudaError_t launch_weight_map_fused(const float* x, float* w, size_t n, int mode, int in_type, float pot_neg_cap,
                                     float pot_drop_x, cudaStream_t stream);
 cudaError_t status_word_address(int** out);
+cudaError_t launch_selftest_wait(int* status, long long limit_cycles, cudaStream_t stream);
 }  // namespace rowmax
 
 namespace {
@@ -283,7 +284,8 @@ int attn_get_schedule(int D, int in_dtype, int weight_mode, int causal, int* til
     return ATTN_OK;
 }
 
-int attn_device_status(void) {
+// Synchronises the device and reads the status word; *code gets the raw word.
+static int read_status_word(int* code) {
     int* word = nullptr;
     int rc = status_word(&word);
     if (rc != ATTN_OK) return rc;
@@ -291,7 +293,34 @@ int attn_device_status(void) {
     cudaError_t e = cudaDeviceSynchronize();
     if (e == cudaSuccess) e = cudaMemcpy(&host, word, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return ATTN_ERR_CUDA; }
-    return host;
+    *code = host;
+    return ATTN_OK;
+}
+
+int attn_device_status(void) {
+    int code = 0;
+    int rc = read_status_word(&code);
+    if (rc != ATTN_OK) return rc;
+    return code != 0 ? ATTN_ERR_TIMEOUT : ATTN_OK;
+}
+
+int attn_device_status_code(void) {
+    int code = 0;
+    int rc = read_status_word(&code);
+    return rc != ATTN_OK ? rc : code;
+}
+
+int attn_selftest_wait(long long limit_cycles, void* stream) {
+    if (limit_cycles <= 0 || limit_cycles > 2000000000LL) return ATTN_ERR_BAD_VALUE;
+    int rc = check_arch();
+    if (rc != ATTN_OK) return rc;
+    int* word = nullptr;
+    rc = status_word(&word);
+    if (rc != ATTN_OK) return rc;
+    cudaError_t e = rowmax::launch_selftest_wait(word, limit_cycles, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { g_last_cuda_error = static_cast<int>(e); return ATTN_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTN_OK;
 }
 
 int attn_device_status_reset(void) {

@@ -31,7 +31,7 @@ struct WsCfg {
     static constexpr int kRingBytes = kSlots * C::kTileBytes;
     static constexpr int kScaleOff = kQBytes + kRingBytes;        // float alpha[2][128]
     static constexpr int kBarOff = kScaleOff + 2 * 128 * 4;
-    static constexpr int kNumBars = 2 * kSlots + 8 * 2;
+    static constexpr int kNumBars = 2 * kSlots + 8 * 2 + 1;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kSmemBytes = kMiscOff + 16 + 1024;       // + manual 1024-byte alignment slack
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
@@ -61,6 +61,7 @@ template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setma
 // tiles' softmax phases apart for the first iterations.
 constexpr bool kStagger = true;
 
+constexpr int kBarSelftest = 0x7F;
 enum BarId : int { kBarQFull = 0, kBarQEmpty = 1, kBarKvFull = 2, kBarKvEmpty = 3, kBarSFull = 4, kBarPFull = 5,
                    kBarOFull = 6, kBarScale = 7, kBarORescaled = 8, kBarOFree = 9 };
 
@@ -117,7 +118,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t bar0 = smem_u32(smem + W::kBarOff);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + W::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + W::kMiscOff + 4);
-    const WaitCtx wctx{abort_flag, p.status};
+    const WaitCtx wctx{abort_flag, p.status, kWaitLimitCycles};
 
     // barrier addresses
     auto bar_kv_full = [&](int s) { return bar0 + 8u * s; };
@@ -131,8 +132,15 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto bar_scale = [&](int t) { return bar_x(5, t); };       // softmax -> correction: alpha_t(j) in smem
     auto bar_o_rescaled = [&](int t) { return bar_x(6, t); };  // correction -> MMA: O_t rescaled for tile j
     auto bar_o_free = [&](int t) { return bar_x(7, t); };      // epilogue -> MMA: O_t has been read out
+    const uint32_t bar_drain = bar0 + 8u * (2 * NS + 16);      // abort path only: the MMA warp's last commit
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = warp >> 2;
+    // The status word is sticky: once a wait has expired (in an earlier launch, or in another CTA of this one) and
+    // until the host clears it, a CTA that starts is a no-op: it touches neither its outputs nor TMEM nor TMA.
+    // One thread reads the word so that the whole CTA takes the same way.
+    if (tid == 0) *abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0);
+    __syncthreads();
+    if (*abort_flag) return;
 #ifdef ROWMAX_TRACE
     const long long trace_t0 = clock64();
 #endif
@@ -159,7 +167,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             mbar_init(bar_o_rescaled(t), 4);  // one arrival per correction warp
             mbar_init(bar_o_free(t), 4);      // one arrival per softmax warp (epilogue)
         }
-        *abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0);
+        mbar_init(bar_drain, 1);
         fence_mbar_init();
     }
     constexpr uint32_t kTmemCols = 512;
@@ -220,6 +228,15 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 }
                 if (it.n_max == 0) load_q(1);
             }
+            // Before the CTA ends every load this thread issued must have landed.  Normally the consumers have
+            // seen to that and these waits return at once; after an expired wait they may have stopped waiting while
+            // copies were still writing shared memory, so wait (bounded) for the last use of every ring slot and
+            // Q buffer.
+            for (int idx = kv_idx > NS ? kv_idx - NS : 0; idx < kv_idx; ++idx)
+                mbar_wait_quiet(bar_kv_full(idx % NS), (idx / NS) & 1, kDrainLimitCycles);
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+                if (q_use[t] > 0) mbar_wait_quiet(bar_q_full(t), (q_use[t] - 1) & 1, kDrainLimitCycles);
         } else if (warp == 12) {
             // ------------------------------------------------------------ MMA issuer
             // The whole warp walks the loop (so addresses and descriptors stay warp-uniform values);
@@ -318,6 +335,10 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     if (it.n[t] > 0) ++q_use[t];
                 }
             }
+            // No MMA of this thread may still be running when TMEM is handed back: one last commit, awaited with a
+            // bound (it arrives at once unless a wait expired and the roles left their loops early).
+            if (leader) umma_commit(bar_drain);
+            mbar_wait_quiet(bar_drain, 0, kDrainLimitCycles);
         }
     } else if (wg == 2) {
         // ---------------------------------------------------------------- correction
@@ -532,7 +553,8 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (q0 < p.Sq) {
                 const bool has_keys = (m_run != -INFINITY) && l_run > 0.f;
                 const float inv = has_keys ? p.v_descale / l_run : 0.f;
-                if (row < p.Sq && p.lse != nullptr) {
+                const bool alive = !*abort_flag;      // after an expired wait the accumulators are not to be trusted: store nothing
+                if (alive && row < p.Sq && p.lse != nullptr) {
                     const float lse = has_keys ? 0.6931471805599453f * (m_run * p.c + log2f(l_run) - p_off) : -INFINITY;
                     p.lse[(static_cast<size_t>(it.b) * p.Hq + it.h) * p.Sq + row] = lse;
                 }
@@ -559,7 +581,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = 0;
                     }
-                    if (row < p.Sq) {
+                    if (alive && row < p.Sq) {
 #pragma unroll
                         for (int v4 = 0; v4 < 4; ++v4) {
                             uint4 pk;
@@ -799,6 +821,26 @@ cudaError_t launch_weight_map(const float* x, float* w, size_t n, int mode, cuda
     size_t blocks = (n + threads - 1) / threads;
     if (blocks > 148 * 8) blocks = 148 * 8;
     weight_map_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(x, w, n, mode, 1u << 22);
+    return cudaGetLastError();
+}
+
+// One warp waits on a barrier nobody arrives on, with a short limit: the wait gives up, records its code in the
+// status word and the kernel returns.  Exercises the bounded-wait path without touching the attention kernels.
+__global__ void selftest_wait_kernel(int* status, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int cta_abort;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        cta_abort = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    const WaitCtx ctx{&cta_abort, status, limit_cycles};
+    mbar_wait(smem_u32(&bar), 0, ctx, (kRoleSelftest << 8) | kBarSelftest);
+}
+
+cudaError_t launch_selftest_wait(int* status, long long limit_cycles, cudaStream_t stream) {
+    selftest_wait_kernel<<<1, 32, 0, stream>>>(status, limit_cycles);
     return cudaGetLastError();
 }
 

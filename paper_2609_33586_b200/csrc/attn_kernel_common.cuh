@@ -43,7 +43,7 @@ struct AttnParams {
 
 // Status codes written by expired waits: role << 8 | barrier id.
 enum : int {
-    kRoleSerial = 1, kRoleLoad = 2, kRoleMma = 3, kRoleSoftmax = 4, kRoleCorr = 5, kRoleEpi = 6
+    kRoleSerial = 1, kRoleLoad = 2, kRoleMma = 3, kRoleSoftmax = 4, kRoleCorr = 5, kRoleEpi = 6, kRoleSelftest = 7
 };
 
 }  // namespace rowmax

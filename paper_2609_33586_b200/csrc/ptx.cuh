@@ -56,21 +56,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 struct WaitCtx {
     volatile int* cta_abort;  // shared memory
     int* global_status;       // global memory
+    long long limit_cycles;   // how long one wait may last
 };
 
 constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second at B200 clocks
 
+// Every turn of the waiting loop looks at the device-global status word.  That load from global memory also keeps
+// the waiting warp away from the barrier for a few hundred clocks per turn, which measured faster than a loop that
+// only polls the barrier and than one that sleeps (those take shared-memory cycles from the tensor cores' operand
+// reads); a quick-polling variant for single hand-offs changed nothing.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx, int code) {
     if (mbar_try_wait(bar, parity)) return;
     if (*ctx.cta_abort) return;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*ctx.cta_abort) return;
-        if (*reinterpret_cast<volatile int*>(ctx.global_status) != 0 || clock64() - t0 > kWaitLimitCycles) {
+        if (*reinterpret_cast<volatile int*>(ctx.global_status) != 0 || clock64() - t0 > ctx.limit_cycles) {
             *ctx.cta_abort = 1;
             atomicCAS(ctx.global_status, 0, code);
             return;
         }
+    }
+}
+
+// Bounded wait of the tear-down path after an expired wait: no status, no abort check, just a limit.
+constexpr long long kDrainLimitCycles = 20000000LL;   // about ten milliseconds
+__device__ __forceinline__ void mbar_wait_quiet(uint32_t bar, uint32_t parity, long long limit_cycles) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > limit_cycles) return;
     }
 }
 
