@@ -43,7 +43,10 @@ METRIC = "attn_fwd_tflops_h15_causal_8k_fp8"
 # dram__bytes_read.sum + dram__bytes_write.sum of one h15 launch on the headline workload, from the ncu
 # capture summarised in profiles/attn_fwd_ws_causal_8k_fp8.txt (algorithmic: 101 MB in + 68 MB out)
 NCU_DRAM_BYTES_PER_LAUNCH = 171.8e6 + 32.6e6
-MODE_IDS = {"exact": 0, "pot": 1, "h15": 2, "h15k2": 3, "h15k3": 4, "exact_poly": 5}
+# weight mode, or (weight mode, eighths of the scores on the polynomial route) for the partly emulated exact control
+MODE_IDS = {"exact": 0, "pot": 1, "h15": 2, "h15k2": 3, "h15k3": 4, "exact_poly": 5,
+            "exact_poly_12": (5, 1), "exact_poly_25": (5, 2), "exact_poly_37": (5, 3), "exact_poly_50": (5, 4)}
+POLY_SHARE = {"exact_poly": 0.25, "exact_poly_12": 0.125, "exact_poly_25": 0.25, "exact_poly_37": 0.375, "exact_poly_50": 0.5}
 N_SMS = 148                   # B200
 MUFU_PER_CLK_PER_SM = 16      # ex2 results per clock per SM (Sec. 1)
 
@@ -67,7 +70,12 @@ def matrix_workloads():
         nm = f"causal_{S // 1024}k_fp8_b1"
         out.append((nm, paper(nm, S, True, "fp8_e4m3"), ("exact", "h15")))
     out.append(("causal_8k_fp8_family", WORKLOADS[2].with_(name="causal_8k_fp8_family", B=1),
-                ("exact", "exact_poly", "pot", "h15", "h15k2", "h15k3")))
+                ("exact", "pot", "h15", "h15k2", "h15k3")))
+    # the stronger exact control: a share of the 2^x on the FMA pipe (App. B "FA4's own parameter space")
+    out.append(("causal_8k_fp8_emulated_exact", WORKLOADS[2].with_(name="causal_8k_fp8_emulated_exact", B=1),
+                ("exact", "exact_poly_12", "exact_poly_25", "exact_poly_37", "exact_poly_50", "h15")))
+    out.append(("causal_8k_bf16_emulated_exact", paper("causal_8k_bf16_emulated_exact", 8192, True, "bf16"),
+                ("exact", "exact_poly_12", "exact_poly_25", "exact_poly_37", "exact_poly_50", "h15")))
     return out
 
 
@@ -253,10 +261,11 @@ class DeviceRun:
         self.o = torch.empty((wl.B, wl.Sq, wl.Hq, wl.D), dtype=torch.bfloat16, device=device)
         self.lse = torch.empty((wl.B, wl.Hq, wl.Sq), dtype=torch.float32, device=device)
 
-    def step(self, mode: int):
+    def step(self, mode):
+        mode, eighths = mode if isinstance(mode, tuple) else (mode, None)
         self.b.attn_fwd(self.q, self.k, self.v, causal=self.wl.causal, softmax_scale=self.wl.softmax_scale,
                         weight_mode=mode, q_descale=self.inp.q_descale, k_descale=self.inp.k_descale,
-                        v_descale=self.inp.v_descale, out=self.o, lse=self.lse)
+                        v_descale=self.inp.v_descale, out=self.o, lse=self.lse, poly_eighths=eighths)
 
     def time_steps(self, mode: int, steps: int, warmup: int) -> float:
         """ms per step: CUDA events on the launching (current) stream around `steps` back-to-back calls."""
@@ -324,8 +333,8 @@ def roofline_entries(res, wl: Workload, peaks):
         m["frac_tensor_burst"] = tf / (ratio * peaks["bf16_tflops"])
         if peaks.get("bf16_tflops_sustained"):
             m["frac_tensor_sustained"] = tf / (ratio * peaks["bf16_tflops_sustained"])
-        if name in ("exact", "exact_poly") and m.get("sm_mhz_median"):
-            share = 0.75 if name == "exact_poly" else 1.0   # a quarter of the scores bypasses the unit
+        if (name == "exact" or name in POLY_SHARE) and m.get("sm_mhz_median"):
+            share = 1.0 - POLY_SHARE.get(name, 0.0)         # the emulated share of the scores bypasses the unit
             bound_ms = 1e3 * share * scores / (MUFU_PER_CLK_PER_SM * N_SMS * m["sm_mhz_median"] * 1e6)
             m["mufu_bound_ms"] = bound_ms
             m["frac_mufu"] = bound_ms / m["ms"]

@@ -118,6 +118,20 @@ int attn_fwd_pot(const void* q, const void* k, const void* v, void* o, float* ls
                  int pot_kmax, int drop_tail, void* stream);
 
 /*
+ * attn_fwd_exact_emulated — attn_fwd in exact mode with share_eighths / 8 of the 2^x evaluated by floor + cubic +
+ * exponent insert on the FMA and integer pipes instead of the special-function unit (relative error <= 1.1e-4):
+ * the partial emulation that the paper's baseline kernel uses, with its share as a parameter (App. B "FA4's own
+ * parameter space": shares 0 to 75 %, the fastest stock setting at 37.5 %).  share_eighths = 1, 2, 3, 4 (12.5, 25,
+ * 37.5, 50 %), else ATTN_ERR_BAD_VALUE; attn_fwd(..., ATTN_W_EXACT_POLY, ...) is share_eighths = 2.  Shares other
+ * than 2 are built for D = 128 and bf16 / fp8 inputs (ATTN_ERR_UNSUPPORTED otherwise).  Same tolerances as exact.
+ */
+int attn_fwd_exact_emulated(const void* q, const void* k, const void* v, void* o, float* lse,
+                            int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                            int causal, float softmax_scale, int in_dtype,
+                            float q_descale, float k_descale, float v_descale,
+                            int share_eighths, void* stream);
+
+/*
  * attn_weight_map — applies the weight map of `weight_mode` to n fp32 offsets with the same device
  * function the fused kernel uses (Eq. m-exact / Eq. rowmax-pot / Eq. h15; the h15 input is clamped
  * below at -126, App. B.1 "Implementation"; inside the fused kernel a key tile that holds masked scores

@@ -20,7 +20,7 @@ MODES = {"exact": W_EXACT, "pot": W_POT, "h15": W_H15, "h15k2": W_H15K2, "h15k3"
 _LIB_PATH = Path(__file__).resolve().parent / "libattn_b200.so"
 _lib = None
 
-EXPORTS = ("attn_fwd", "attn_fwd_tau", "attn_fwd_pot", "attn_weight_map", "attn_weight_map_pot", "attn_weight_map_fused", "attn_get_schedule", "attn_device_status",
+EXPORTS = ("attn_fwd", "attn_fwd_tau", "attn_fwd_pot", "attn_fwd_exact_emulated", "attn_weight_map", "attn_weight_map_pot", "attn_weight_map_fused", "attn_get_schedule", "attn_device_status",
            "attn_device_status_code", "attn_selftest_wait", "attn_device_status_reset", "attn_launch_count", "attn_status_string",
            "attn_last_cuda_error", "attn_version")
 
@@ -46,6 +46,8 @@ def lib() -> ctypes.CDLL:
         L.attn_fwd_tau.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, i, f, f, f, f, vp]
         L.attn_fwd_pot.restype = i
         L.attn_fwd_pot.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, f, f, f, i, i, vp]
+        L.attn_fwd_exact_emulated.restype = i
+        L.attn_fwd_exact_emulated.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, f, f, f, i, vp]
         L.attn_weight_map.restype = i
         L.attn_weight_map.argtypes = [vp, vp, ctypes.c_size_t, i, vp]
         L.attn_weight_map_pot.restype = i
@@ -133,9 +135,14 @@ def in_dtype_of(t: torch.Tensor) -> int:
 
 def attn_fwd_raw(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale,
                  weight_mode, in_dtype, q_descale, k_descale, v_descale, stream_ptr, rescale_tau=None,
-                 pot_tail=None) -> int:
+                 pot_tail=None, poly_eighths=None) -> int:
     """Direct call with integer device addresses; returns the status code.  With `rescale_tau` the
-    call goes to attn_fwd_tau, with `pot_tail` = (K_max, drop_tail) to attn_fwd_pot."""
+    call goes to attn_fwd_tau, with `pot_tail` = (K_max, drop_tail) to attn_fwd_pot, with `poly_eighths`
+    to attn_fwd_exact_emulated."""
+    if poly_eighths is not None:
+        return lib().attn_fwd_exact_emulated(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
+                                             softmax_scale, in_dtype, q_descale, k_descale, v_descale,
+                                             int(poly_eighths), stream_ptr)
     if pot_tail is not None:
         return lib().attn_fwd_pot(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, int(causal),
                                   softmax_scale, in_dtype, q_descale, k_descale, v_descale,
@@ -152,11 +159,14 @@ def attn_fwd_raw(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D, cau
 def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool, softmax_scale: float,
              weight_mode: int, q_descale: float = 1.0, k_descale: float = 1.0, v_descale: float = 1.0,
              out: torch.Tensor | None = None, lse: torch.Tensor | None = None, return_lse: bool = True,
-             rescale_tau: float | None = None, pot_tail=None, stream=None):
+             rescale_tau: float | None = None, pot_tail=None, poly_eighths=None, stream=None):
     """q (B,Sq,Hq,D), k/v (B,Sk,Hkv,D): contiguous CUDA tensors, bf16, float16 or float8_e4m3fn.
     Returns (O bf16 (B,Sq,Hq,D), LSE fp32 (B,Hq,Sq) or None).  `rescale_tau` (bf16 inputs only) selects
     the deferred-rescale entry point attn_fwd_tau; `pot_tail` = (K_max, drop_tail) selects attn_fwd_pot
-    (Rowmax-PoT with that tail; `weight_mode` must then be W_POT)."""
+    (Rowmax-PoT with that tail; `weight_mode` must then be W_POT); `poly_eighths` (1..4) selects
+    attn_fwd_exact_emulated (`weight_mode` must then be W_EXACT_POLY)."""
+    if poly_eighths is not None and weight_mode != W_EXACT_POLY:
+        raise ValueError("poly_eighths goes with weight_mode = W_EXACT_POLY")
     if pot_tail is not None and weight_mode != W_POT:
         raise ValueError("pot_tail goes with weight_mode = W_POT")
     for t in (q, k, v):
@@ -176,7 +186,7 @@ def attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, causal: bool,
     rc = attn_fwd_raw(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                       lse.data_ptr() if lse is not None else None, B, Hq, Hkv, Sq, Sk, D, causal,
                       softmax_scale, weight_mode, dt, q_descale, k_descale, v_descale,
-                      _stream_ptr(stream), rescale_tau, pot_tail)
+                      _stream_ptr(stream), rescale_tau, pot_tail, poly_eighths)
     if rc != 0:
         raise AttnError(rc, "attn_fwd")
     return out, lse

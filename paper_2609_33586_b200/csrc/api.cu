@@ -127,7 +127,8 @@ namespace {
 // Every forward entry point ends here.  pot_kmax / pot_drop_tail matter in ATTN_W_POT mode only.
 int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
              int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
-             float k_descale, float v_descale, float rescale_tau, int pot_kmax, int pot_drop_tail, void* stream) {
+             float k_descale, float v_descale, float rescale_tau, int pot_kmax, int pot_drop_tail, int poly_eighths,
+             void* stream) {
     if (!q || !k || !v || !o) return ATTN_ERR_NULLPTR;
     if (weight_mode < ATTN_W_EXACT || weight_mode > ATTN_W_EXACT_POLY) return ATTN_ERR_BAD_ENUM;
     if (in_dtype != ATTN_IN_BF16 && in_dtype != ATTN_IN_FP8_E4M3 && in_dtype != ATTN_IN_FP16) return ATTN_ERR_BAD_ENUM;
@@ -185,7 +186,12 @@ int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, i
 
     static_assert(ATTN_IN_BF16 == rowmax::kInBF16 && ATTN_IN_FP8_E4M3 == rowmax::kInFP8 && ATTN_IN_FP16 == rowmax::kInFP16,
                   "the kernel's storage-type codes are those of the C interface");
-    const int kernel_mode = (weight_mode == ATTN_W_POT && drop) ? rowmax::kPotDrop : weight_mode;
+    int kernel_mode = (weight_mode == ATTN_W_POT && drop) ? rowmax::kPotDrop : weight_mode;
+    if (weight_mode == ATTN_W_EXACT_POLY) {
+        if (poly_eighths < 1 || poly_eighths > 4) return ATTN_ERR_BAD_VALUE;
+        const int by_share[5] = {0, rowmax::kExactPoly1, rowmax::kExactPoly, rowmax::kExactPoly3, rowmax::kExactPoly4};
+        kernel_mode = by_share[poly_eighths];
+    }
     cudaError_t e = rowmax::launch_attn_fwd(D, in_dtype, kernel_mode, tq, tk, tv, p, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(e);
@@ -203,14 +209,21 @@ int attn_fwd_tau(const void* q, const void* k, const void* v, void* o, float* ls
                  int Sk, int D, int causal, float softmax_scale, int weight_mode, int in_dtype, float q_descale,
                  float k_descale, float v_descale, float rescale_tau, void* stream) {
     return fwd_impl(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale, weight_mode, in_dtype, q_descale,
-                    k_descale, v_descale, rescale_tau, ATTN_POT_KMAX_DEFAULT, 0, stream);
+                    k_descale, v_descale, rescale_tau, ATTN_POT_KMAX_DEFAULT, 0, 2, stream);
+}
+
+int attn_fwd_exact_emulated(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
+                            int Sq, int Sk, int D, int causal, float softmax_scale, int in_dtype, float q_descale,
+                            float k_descale, float v_descale, int share_eighths, void* stream) {
+    return fwd_impl(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale, ATTN_W_EXACT_POLY, in_dtype, q_descale,
+                    k_descale, v_descale, 0.0f, ATTN_POT_KMAX_DEFAULT, 0, share_eighths, stream);
 }
 
 int attn_fwd_pot(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
                  int Sk, int D, int causal, float softmax_scale, int in_dtype, float q_descale, float k_descale,
                  float v_descale, int pot_kmax, int drop_tail, void* stream) {
     return fwd_impl(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, causal, softmax_scale, ATTN_W_POT, in_dtype, q_descale,
-                    k_descale, v_descale, 0.0f, pot_kmax, drop_tail, stream);
+                    k_descale, v_descale, 0.0f, pot_kmax, drop_tail, 2, stream);
 }
 
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,

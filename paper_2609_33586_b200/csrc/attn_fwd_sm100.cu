@@ -500,7 +500,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         weights_chunk32<FP8, MODE, false, true, HALF, true>(s[cc], rs, 32, acc, pw);
                         tmem_st16(tS + cc * 16, pw);
                     }
-                } else if ((is_pot(MODE) || MODE == kExactPoly) && masked_tile) {
+                } else if (is_pot(MODE) && masked_tile) {
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t pw[16];
@@ -655,6 +655,14 @@ static cudaError_t dispatch_mode(int mode, const CUtensorMap& tq, const CUtensor
             case kH15K3: return launch_ws<D, IN, kH15K3>(tq, tk, tv, p, stream);
             case kExactPoly: return launch_ws<D, IN, kExactPoly>(tq, tk, tv, p, stream);
             default: break;
+        }
+        if constexpr (D == 128) {   // the other emulation shares: the paper's main head dimension only
+            switch (mode) {
+                case kExactPoly1: return launch_ws<D, IN, kExactPoly1>(tq, tk, tv, p, stream);
+                case kExactPoly3: return launch_ws<D, IN, kExactPoly3>(tq, tk, tv, p, stream);
+                case kExactPoly4: return launch_ws<D, IN, kExactPoly4>(tq, tk, tv, p, stream);
+                default: break;
+            }
         }
     }
     return cudaErrorInvalidValue;

@@ -12,10 +12,17 @@ constexpr int kTileN = 128;  // keys per tile
 enum InType : int { kInBF16 = 0, kInFP8 = 1, kInFP16 = 2 };
 // kPotDrop is internal: Rowmax-PoT with a dropped tail (the C interface selects it through attn_fwd_pot), a
 // separate instance so that the clamped tail does not pay for the comparison that drops.
-enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4, kExactPoly = 5, kPotDrop = 6 };
+// kExactPoly1/3/4 are internal too: the partly emulated exact mode with 1, 3 or 4 eighths of the scores on the
+// polynomial route (kExactPoly itself: 2 eighths), selected through attn_fwd_exact_emulated.
+enum WeightMode : int { kExact = 0, kPot = 1, kH15 = 2, kH15K2 = 3, kH15K3 = 4, kExactPoly = 5, kPotDrop = 6,
+                        kExactPoly1 = 7, kExactPoly3 = 8, kExactPoly4 = 9 };
+// eighths of the scores whose 2^x is evaluated by the polynomial instead of the special-function unit (0: none)
+__host__ __device__ constexpr int exact_poly_eighths(int mode) {
+    return mode == kExactPoly ? 2 : mode == kExactPoly1 ? 1 : mode == kExactPoly3 ? 3 : mode == kExactPoly4 ? 4 : 0;
+}
 __host__ __device__ constexpr bool is_pot(int mode) { return mode == kPot || mode == kPotDrop; }
 // modes whose weight is 2^x itself (with the P offset folded into x)
-__host__ __device__ constexpr bool is_exact_like(int mode) { return mode == kExact || mode == kExactPoly; }
+__host__ __device__ constexpr bool is_exact_like(int mode) { return mode == kExact || exact_poly_eighths(mode) > 0; }
 // input-rounding exponent of the h15 family member: steps of 2^-k octaves (0: not a family member)
 __host__ __device__ constexpr int h15_family_k(int mode) {
     return mode == kH15 ? 1 : mode == kH15K2 ? 2 : mode == kH15K3 ? 3 : 0;

@@ -219,9 +219,11 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             t.x = fmaf(fma_sat(sv.x, rs.su, rs.ou), rs.sat_mul, kH15Magic);
             t.y = fmaf(fma_sat(sv.y, rs.su, rs.ou), rs.sat_mul, kH15Magic);
             w = h15_weight_pair_from_t<kOff, h15_family_k(MODE)>(t, rs.two22);
-        } else if constexpr (MODE == kExactPoly && !MASKED) {
-            // every fourth pair (25 % of the scores) takes the polynomial route, the rest the hardware ex2
-            if (i % 4 == 3) {
+        } else if constexpr (exact_poly_eighths(MODE) > 0) {
+            // e eighths of the pairs, spread evenly, take the polynomial route, the rest the hardware ex2; a masked
+            // score (-inf) weighs nothing on either route
+            constexpr int e = exact_poly_eighths(MODE);
+            if (((i * e) & 7) < e) {
                 w.x = w_exact_poly3(x.x);
                 w.y = w_exact_poly3(x.y);
             } else {

@@ -19,9 +19,11 @@ __device__ __forceinline__ float w_exact(float x) {
 // round-down add of 2^23 + 2^22, a cubic for 2^f on the fraction f in [0,1), and floor(x) added to the
 // exponent field.  The cubic is this build's own fit: it interpolates 2^0 and 2^1 (so the map is continuous
 // across octaves) and minimises the largest relative error on [0,1], which is 1.03e-4.
-// Valid for -126 <= x < 127; smaller inputs are clamped, so the result is never exactly zero.
+// Valid for -127 <= x < 127; smaller inputs (a masked score is -inf) are clamped at -127, where floor = -127 and
+// fraction = 0 give the exponent field 0 and the fraction 0: exactly +0, as the hardware ex2 with flush-to-zero
+// gives.  Between -127 and -126 the result is a denormal pattern (2^-127 (1 + f) read as a fraction), below 2^-126.
 __device__ __forceinline__ float w_exact_poly3(float x) {
-    x = fmaxf(x, -126.0f);
+    x = fmaxf(x, -127.0f);
     const float t = __fadd_rd(x, 12582912.0f);   // 2^23 + 2^22 + floor(x), exact
     const float f = x - (t - 12582912.0f);       // fraction in [0,1)
     const float p = fmaf(fmaf(fmaf(0.07826797f, f, 0.22630768f), f, 0.69542432f), f, 1.0f);   // 2^f in [1,2]

@@ -66,6 +66,42 @@ def test_partly_emulated_exact_mode_meets_the_exact_tolerances(wl):
     assert st["ok"], st
 
 
+@pytest.mark.parametrize("eighths", [1, 2, 3, 4])
+@pytest.mark.parametrize("wl", [
+    Workload("share_bf16", 2, 4, 2, 300, 428, 128, True, "bf16", 57),
+    Workload("share_fp8", 1, 2, 2, 384, 384, 128, True, "fp8_e4m3", 58),
+], ids=lambda w: w.name)
+def test_emulation_share_of_the_exact_control(wl, eighths):
+    # 12.5 to 50 % of the exponentials on the polynomial route: the exact tolerances hold for every share
+    inp = make_inputs(wl)
+    q, k, v = inp.q.cuda(), inp.k.cuda(), inp.v.cuda()
+    o, lse = binding.attn_fwd(q, k, v, causal=wl.causal, softmax_scale=wl.softmax_scale, weight_mode=EXACT_POLY,
+                              q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale, poly_eighths=eighths)
+    ref_o, ref_lse = binding.attn_fwd(q, k, v, causal=wl.causal, softmax_scale=wl.softmax_scale, weight_mode=orc.W_EXACT,
+                                      q_descale=inp.q_descale, k_descale=inp.k_descale, v_descale=inp.v_descale)
+    torch.cuda.synchronize()
+    from parity_util import run_oracle, TOL
+    ref = run_oracle(wl, inp, orc.W_EXACT)
+    got = o.float().cpu().numpy().transpose(0, 2, 1, 3)
+    tol = TOL[wl.in_dtype]["o_max"] * (2.0 if wl.in_dtype == "fp8_e4m3" else 1.0)   # causal rows with few keys: see parity_util
+    assert np.abs(got - ref["O"]).max() <= tol
+    assert np.abs(lse.cpu().numpy() - ref["LSE"]).max() <= 1e-3
+    # and close to the plain exact mode of the same kernel
+    assert (o.float() - ref_o.float()).abs().max().item() <= tol
+    assert (lse - ref_lse).abs().max().item() <= 5e-4
+
+
+def test_emulation_share_limits():
+    q = torch.zeros(1, 128, 2, 64, dtype=torch.bfloat16, device="cuda")
+    args = (q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 1, 2, 2, 128, 128)
+    tail = (1, 0.1, EXACT_POLY, binding.IN_BF16, 1.0, 1.0, 1.0, None)
+    assert binding.attn_fwd_raw(*args, 64, *tail, poly_eighths=3) == -8       # other shares: D = 128 only
+    assert binding.attn_fwd_raw(*args, 64, *tail, poly_eighths=2) == 0
+    assert binding.attn_fwd_raw(*args, 64, *tail, poly_eighths=5) == -9
+    assert binding.attn_fwd_raw(*args, 64, *tail, poly_eighths=0) == -9
+    torch.cuda.synchronize()
+
+
 def test_partly_emulated_exact_mode_full_size_8k_fp8():
     wl = WORKLOADS[2]
     st = compare(wl, EXACT_POLY, rows=_sample_rows(wl.Sq, 127))

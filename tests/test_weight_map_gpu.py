@@ -53,6 +53,8 @@ def test_emulated_exact_map_is_within_its_stated_error():
     assert np.all(np.diff(got[np.argsort(x, kind="stable")]) >= 0)          # monotone, continuous across octaves
     ints = np.arange(-126, 17, dtype=np.float32)
     assert np.array_equal(_gpu_map(ints, binding.W_EXACT_POLY), np.exp2(ints.astype(np.float64)).astype(np.float32))
+    # a masked score (-inf) and anything below -127 weigh exactly nothing, as with the hardware ex2
+    assert _gpu_map(np.array([-np.inf, -127.0, -200.0], np.float32), binding.W_EXACT_POLY).tolist() == [0.0, 0.0, 0.0]
 
 
 def test_in_place_and_empty():
