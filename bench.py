@@ -42,7 +42,7 @@ TWIN = WORKLOADS[3]           # non-causal 8K fp8
 METRIC = "attn_fwd_tflops_h15_causal_8k_fp8"
 # dram__bytes_read.sum + dram__bytes_write.sum of one h15 launch on the headline workload, from the ncu
 # capture summarised in profiles/attn_fwd_ws_causal_8k_fp8.txt (algorithmic: 101 MB in + 68 MB out)
-NCU_DRAM_BYTES_PER_LAUNCH = 171.8e6 + 32.6e6
+NCU_DRAM_BYTES_PER_LAUNCH = 171.1e6 + 32.1e6
 # weight mode, or (weight mode, eighths of the scores on the polynomial route) for the partly emulated exact control
 MODE_IDS = {"exact": 0, "pot": 1, "h15": 2, "h15k2": 3, "h15k3": 4, "exact_poly": 5,
             "exact_poly_12": (5, 1), "exact_poly_25": (5, 2), "exact_poly_37": (5, 3), "exact_poly_50": (5, 4)}

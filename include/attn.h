@@ -135,7 +135,9 @@ int attn_fwd_exact_emulated(const void* q, const void* k, const void* v, void* o
  * attn_weight_map — applies the weight map of `weight_mode` to n fp32 offsets with the same device
  * function the fused kernel uses (Eq. m-exact / Eq. rowmax-pot / Eq. h15; the h15 input is clamped
  * below at -126, App. B.1 "Implementation"; inside the fused kernel a key tile that holds masked scores
- * clamps at -127 instead, the input whose weight pattern is +0, so that a masked key weighs nothing).  x and w are device arrays of n floats; they may alias.
+ * clamps at -127 instead, the input whose weight pattern is +0, so that a masked key weighs nothing; on fp8 inputs, whose weights
+ * carry a 2^15 offset, that pattern is 2^-112: zero in P, and below one part in 2^127 of a row sum).  x and w are device arrays
+ * of n floats; they may alias.
  * pot and h15 results are bit-exact by definition; exact uses the hardware ex2 approximation with
  * subnormal results flushed to zero.
  */

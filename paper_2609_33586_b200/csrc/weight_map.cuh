@@ -57,7 +57,9 @@ __device__ __forceinline__ float w_h15_doubled(float x2) { return h15_weight_fro
 // shift) for the fp8 P formats.  kClamp = false skips the clamp; the caller must know that both
 // inputs are at or above -126 * 2^K.  The clamp value is -126 * 2^K (Eq. h15: the weight floor 2^-126);
 // the fused kernel passes -127 * 2^K in a key tile that holds masked scores: that input gives the
-// bit pattern of +0 (times 2^kOff), so a masked score (-inf) weighs exactly nothing.
+// bit pattern of +0 when kOff = 0 (16-bit inputs): a masked score (-inf) then weighs exactly nothing.  With the fp8
+// P offset (kOff = 15) the pattern is 2^(kOff - 127) = 2^-112 instead: P, which is what multiplies V, still rounds to
+// zero, and the row sum takes 2^-112 against terms of at least 2^15, below one part in 2^127.
 // Two rounded patterns t = 2^23 + 2^22 + n (as floats) -> the two weights (1 + (n mod 2^K) / 2^K) 2^floor(n / 2^K)
 // times 2^kOff: (bits << (23 - K)) + bias, one lane by shift-add (ALU pipe), the other by the equivalent integer
 // multiply-add (FMA pipe).
