@@ -467,10 +467,20 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
                 const float alpha = ex2_approx((m_run - m_use) * p.c);
                 m_run = m_new;
-                sScale[t * 128 + r] = alpha;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_scale(t));
-                if (r == 0) ROWMAX_STAMP(t, j, 2);
+                // exact-like modes post the rescale factor after the first 32 weights are under way, so that its
+                // special-function latency, the shared-memory store and the arrival hide behind them (measured +2 %);
+                // their weight phase is long enough for the correction warps to rescale O in what is left of it.  The
+                // rounding maps post it at once: their weight phase is shorter, and posting late put the correction on
+                // the critical path (measured 5 to 8 % slower).
+                constexpr bool kPostLate = is_exact_like(MODE);
+                auto post_alpha_now = [&]() {
+                    sScale[t * 128 + r] = alpha;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_scale(t));
+                    if (r == 0) ROWMAX_STAMP(t, j, 2);
+                };
+                auto post_alpha = [&]() { if constexpr (kPostLate) post_alpha_now(); };
+                if constexpr (!kPostLate) post_alpha_now();
 
                 // exact: x = s*c - m*c + P offset;  h15 family: scaled input 2^K x = s*(2^K c) - m*(2^K c);  pot: x = s*c - m*c
                 RowScale rs;
@@ -499,6 +509,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         uint32_t pw[16];
                         weights_chunk32<FP8, MODE, false, true, HALF, true>(s[cc], rs, 32, acc, pw);
                         tmem_st16(tS + cc * 16, pw);
+                        if (cc == 0) post_alpha();
                     }
                 } else if (is_pot(MODE) && masked_tile) {
 #pragma unroll
@@ -507,6 +518,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         weights_chunk32<FP8, MODE, true, true, HALF>(s[cc], rs, col_limit - cc * 32, acc, pw);
                         if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                         else tmem_st16(tS + cc * 16, pw);
+                        if (cc == 0) post_alpha();
                     }
                 } else {
                     // h15: the clamp is a no-op unless some score of the warp's rows lies more than 126 octaves
@@ -528,6 +540,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                             weights_chunk32<FP8, MODE, false, true, HALF>(s[cc], rs, 32, acc, pw);
                             if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                             else tmem_st16(tS + cc * 16, pw);
+                            if (cc == 0) post_alpha();
                         }
                     } else {
 #pragma unroll
@@ -536,6 +549,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                             weights_chunk32<FP8, MODE, false, false, HALF>(s[cc], rs, 32, acc, pw);
                             if constexpr (FP8) tmem_st8(tS + cc * 8, pw);
                             else tmem_st16(tS + cc * 16, pw);
+                            if (cc == 0) post_alpha();
                         }
                     }
                 }
