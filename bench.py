@@ -61,7 +61,7 @@ def matrix_workloads():
         ("noncausal_8k_bf16", paper("noncausal_8k_bf16", 8192, False, "bf16"), ("exact", "h15")),
         ("causal_8k_fp16", paper("causal_8k_fp16", 8192, True, "fp16"), ("exact", "h15")),
         ("gqa_causal_2k_bf16", WORKLOADS[1], ("exact", "h15")),
-        ("causal_16k_gqa_bf16", WORKLOADS[4], ("exact", "pot", "h15")),
+        ("causal_16k_gqa_bf16", WORKLOADS[4].with_(name="causal_16k_gqa_bf16"), ("exact", "pot", "h15")),
         ("causal_16k_gqa_fp8", WORKLOADS[4].with_(name="causal_16k_gqa_fp8", in_dtype="fp8_e4m3"), ("exact", "pot", "h15")),
         ("causal_8k_bf16_d64", paper("causal_8k_bf16_d64", 8192, True, "bf16", D=64), ("exact", "h15")),
         ("causal_8k_fp8_d64", paper("causal_8k_fp8_d64", 8192, True, "fp8_e4m3", D=64), ("exact", "h15")),
