@@ -126,16 +126,21 @@ class ClockSampler:
             self._nvml = None
 
     def _sample_nvml(self):
+        # the SM clock every time; power and the throttle reasons every fourth time (each query costs about a
+        # millisecond, and a timed region may last only a few tens of them)
         n = self._nvml
         sm = float(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_SM))
-        pw = n.nvmlDeviceGetPowerUsage(self._h) / 1000.0
-        r = n.nvmlDeviceGetCurrentClocksEventReasons(self._h) if hasattr(n, "nvmlDeviceGetCurrentClocksEventReasons") \
-            else n.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
-        flags = []
-        for name, bit in (("hw_slowdown", 0x8), ("sw_power_cap", 0x4), ("sw_thermal_slowdown", 0x20),
-                          ("hw_thermal_slowdown", 0x40)):
-            if r & bit:
-                flags.append(name)
+        if len(self.samples) % 4 == 0 or not self.samples:
+            pw = n.nvmlDeviceGetPowerUsage(self._h) / 1000.0
+            r = n.nvmlDeviceGetCurrentClocksEventReasons(self._h) if hasattr(n, "nvmlDeviceGetCurrentClocksEventReasons") \
+                else n.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+            flags = []
+            for name, bit in (("hw_slowdown", 0x8), ("sw_power_cap", 0x4), ("sw_thermal_slowdown", 0x20),
+                              ("hw_thermal_slowdown", 0x40)):
+                if r & bit:
+                    flags.append(name)
+        else:
+            pw, flags = self.samples[-1][1], self.samples[-1][2]
         self.samples.append((sm, pw, flags))
 
     def _sample_smi(self):
@@ -157,7 +162,7 @@ class ClockSampler:
                     self._sample_smi()
             except Exception:
                 pass
-            self._stop.wait(0.002 if self._nvml is not None else 0.05)
+            self._stop.wait(0.0005 if self._nvml is not None else 0.05)
 
     def __enter__(self):
         self._thr = threading.Thread(target=self._run, daemon=True)
