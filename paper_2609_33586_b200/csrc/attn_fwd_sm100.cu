@@ -206,20 +206,24 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     for (int bx = 0; bx < C::kBoxes; ++bx)
                         tma_load_4d(dst + bx * C::kBoxBytes, tm, bar, bx * C::kBoxElems, head, row0, it.b);
                 };
+                // After an expired wait nothing more is loaded: a wait then returns at once, and a copy into a buffer
+                // whose last copy may still be under way would leave more in flight than the waits below account for.
                 auto load_q = [&](int t) {
                     if (it.n[t] > 0) {
                         mbar_wait(bar_q_empty(t), (q_use[t] & 1) ^ 1, wctx, (kRoleLoad << 8) | kBarQEmpty);
+                        if (*abort_flag) return;
                         load_tile(&tmQ, sQ + t * C::kTileBytes, bar_q_full(t), it.h, it.q0[t]);
                         ++q_use[t];
                     }
                 };
                 if (round == 0) ROWMAX_STAMP(3, 63, 0);
                 load_q(0);
-                for (int j = 0; j < it.n_max; ++j) {
+                for (int j = 0; j < it.n_max && !*abort_flag; ++j) {
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const int slot = kv_idx % NS, use = kv_idx / NS;
                         mbar_wait(bar_kv_empty(slot), (use & 1) ^ 1, wctx, (kRoleLoad << 8) | kBarKvEmpty);
+                        if (*abort_flag) break;
                         load_tile(kv == 0 ? &tmK : &tmV, sRing + slot * C::kTileBytes, bar_kv_full(slot), it.hk,
                                   j * kTileN);
                         ++kv_idx;
@@ -294,7 +298,9 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     if (leader) umma_commit(bar_kv_empty(kv_base % NS));
                     for (int j = 0; j < it.n_max; ++j) {
                         // Everything the next MMAs need besides P is awaited first (it is normally there long
-                        // before), so that once P_t(j) arrives the P V and next-S MMAs go out back to back.
+                        // before), so that once P_t(j) arrives the P V and next-S MMAs go out back to back.  (The flag
+                        // is read here, off that path: if one of the waits below expires, this step's MMAs still go
+                        // out, on stale operands; nothing is stored after that and the MMAs are awaited at the end.)
                         const bool ok = !*abort_flag;
                         wait_full(kv_base + 2 * j + 1);
                         if (j + 1 < it.n_max) wait_full(kv_base + 2 * j + 2);
