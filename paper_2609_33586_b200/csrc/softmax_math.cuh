@@ -101,6 +101,17 @@ __device__ __forceinline__ uint32_t pack_f16x2_rn(float lo, float hi) {
     return r;
 }
 
+// Four fp32 values to four e5m2 bytes (first argument in the lowest byte) in one instruction.  The instruction rounds
+// stochastically on the random bits it is given; every weight that goes through it here is a lattice weight, exactly
+// representable in e5m2 (a power of two times 1, 1.25, 1.5 or 1.75) down to the format's subnormal grid, so the
+// result does not depend on those bits; with the bits zero a value below that grid is cut off toward zero, as the
+// upper byte of its fp16 pattern would be.
+__device__ __forceinline__ uint32_t pack_e5m2x4_exact(float b0, float b1, float b2, float b3) {
+    uint32_t d;
+    asm("cvt.rs.satfinite.e5m2x4.f32 %0, {%1, %2, %3, %4}, %5;" : "=r"(d) : "f"(b3), "f"(b2), "f"(b1), "f"(b0), "r"(0u));
+    return d;
+}
+
 // Row maximum of 128 scores held as 4 x 32 registers.
 __device__ __forceinline__ float row_max128(const uint32_t (&s)[4][32]) {
     float m[8];
@@ -208,6 +219,7 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
                                                 float2 (&acc)[2], uint32_t* pw) {
     constexpr int kOff = PFormat<FP8, MODE>::kOffLog2;
     uint32_t half16[16];
+    float2 w_even = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const float2 sv = make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
@@ -255,13 +267,21 @@ __device__ __forceinline__ void weights_chunk32(const uint32_t (&s)[32], const R
             if constexpr (is_exact_like(MODE)) pw[i] = pack_bf16_rn(w.x, w.y);
             else pw[i] = __byte_perm(__float_as_uint(w.x), __float_as_uint(w.y), 0x7632);  // exact: at most 3 fraction bits
         } else {
-            if constexpr (PFormat<FP8, MODE>::kE4M3) half16[i] = pack_e4m3x2(w.x, w.y);
-            else half16[i] = pack_f16x2_rn(w.x, w.y);  // at most 2 fraction bits: exact in fp16
+            if constexpr (PFormat<FP8, MODE>::kE4M3) {
+                half16[i] = pack_e4m3x2(w.x, w.y);
+            } else if constexpr (is_pot(MODE)) {
+                // e5m2 P of powers of two: four of them convert exactly at once (measured 2.5 % faster for pot than
+                // the route below, 0.6 % slower for the h15 family, whose pipe mix differs)
+                if (i & 1) pw[i >> 1] = pack_e5m2x4_exact(w_even.x, w_even.y, w.x, w.y);
+                else w_even = w;
+            } else {
+                half16[i] = pack_f16x2_rn(w.x, w.y);  // at most 2 fraction bits: exact in fp16
+            }
         }
     }
-    if constexpr (FP8) {
-        // e4m3 P: two converted pairs per word.  e5m2 P: e5m2 is the upper byte of an fp16 pattern, and these
-        // weights have at most two fraction bits, so the upper bytes of the four halves are the exact P bytes.
+    if constexpr (FP8 && (PFormat<FP8, MODE>::kE4M3 || !is_pot(MODE))) {
+        // e4m3 P: two converted pairs per word.  e5m2 P of the h15 family: e5m2 is the upper byte of an fp16 pattern,
+        // and these weights have at most two fraction bits, so the upper bytes of the four halves are the exact P bytes.
 #pragma unroll
         for (int i = 0; i < 8; ++i)
             pw[i] = __byte_perm(half16[2 * i], half16[2 * i + 1], PFormat<FP8, MODE>::kE4M3 ? 0x5410 : 0x7531);
